@@ -1,0 +1,210 @@
+/*
+ * CPU oracle for the budgeted KV-cache eviction step and the decode attention
+ * that follows it (ForesightKV inference path).
+ *
+ * THIS IS TEST INFRASTRUCTURE.  It is a plain, slow, step-by-step statement of
+ * what the path computes, written from the paper's definitions, in double
+ * precision.  Only the tests, the smoke check and the benchmark's CPU-baseline
+ * leg may call it.  It shares no code with the CUDA library and neither
+ * includes the other.
+ *
+ * Steps (one "segment" = the cache of one sequence, layer and KV head):
+ *   score    Appendix B.1, Eq. "phi_n = sigma(x_n W1 + b1) W2 + b2" with
+ *            x_n = Concat(k_n, v_n, a_n)              (Section 3.1, first equation)
+ *   select   Section 3.1: keep the most recent R pairs, prune the others to
+ *            B - R by keeping the highest scores (the pairs with the lowest
+ *            scores are the ones evicted); deterministic Top-K variant of
+ *            the ablation table on sampling strategies
+ *   compact  Section 3.1: s' = s \ D  (the retained pairs, original order)
+ *   attend   Appendix A, problem set-up: softmax renormalised over the
+ *            retained set S, o = sum_{i in S} a_i v_i
+ *
+ * Parity status: the scorer ARCHITECTURE is pinned (shapes, order k|v|a, the
+ * two affine maps); agreement with the authors' trained checkpoints is
+ * "parity unpinned" - the paper prints no worked numeric example and no
+ * weights.  Everything else is pinned by brute force, closed forms, library
+ * routines and the paper's own identity and error bound (see tests).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ACT_RELU = 0, ACT_SILU = 1, ACT_GELU_TANH = 2, ACT_SIGMOID = 3 };
+
+static double bf16_to_double(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+/* double -> float (round to nearest) -> bf16 (round to nearest even). */
+static uint16_t double_to_bf16(double x) {
+  float f = (float)x;
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u); /* NaN stays NaN */
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7fffu + lsb;
+  return (uint16_t)(u >> 16);
+}
+
+static double activation(double z, int act) {
+  switch (act) {
+    case ACT_RELU: return z > 0.0 ? z : 0.0;
+    case ACT_SILU: return z / (1.0 + exp(-z));
+    case ACT_GELU_TANH: return 0.5 * z * (1.0 + tanh(0.7978845608028654 * (z + 0.044715 * z * z * z)));
+    case ACT_SIGMOID: return 1.0 / (1.0 + exp(-z));
+  }
+  return NAN;
+}
+
+/*
+ * Scorer (Appendix B.1).  K, V: [n][D] bf16 bit patterns; A: [n][F] fp32;
+ * W1: [(2D+F)][H] row-major, rows ordered k | v | a; b1, W2: [H]; phi: [n].
+ */
+void fkv_oracle_score(const uint16_t *K, const uint16_t *V, const float *A, int n, int D, int F, int H,
+                      const float *W1, const float *b1, const float *W2, float b2, int act, float *phi) {
+  for (int i = 0; i < n; ++i) {
+    double out = (double)b2;
+    for (int j = 0; j < H; ++j) {
+      double z = (double)b1[j];
+      for (int c = 0; c < D; ++c) z += bf16_to_double(K[(size_t)i * D + c]) * (double)W1[(size_t)c * H + j];
+      for (int c = 0; c < D; ++c) z += bf16_to_double(V[(size_t)i * D + c]) * (double)W1[(size_t)(D + c) * H + j];
+      for (int c = 0; c < F; ++c) z += (double)A[(size_t)i * F + c] * (double)W1[(size_t)(2 * D + c) * H + j];
+      out += activation(z, act) * (double)W2[j];
+    }
+    phi[i] = (float)out;
+  }
+}
+
+/* Ordering value of a score: -0 counts as +0 and NaN as -infinity. */
+static float canonical(float s) {
+  if (s != s) return -INFINITY;
+  if (s == 0.0f) return 0.0f;
+  return s;
+}
+
+typedef struct { float score; int32_t slot; } ranked_t;
+
+/* Higher score first; equal scores: lower slot first. */
+static int by_score_then_slot(const void *pa, const void *pb) {
+  const ranked_t *a = (const ranked_t *)pa, *b = (const ranked_t *)pb;
+  if (a->score > b->score) return -1;
+  if (a->score < b->score) return 1;
+  return (a->slot > b->slot) - (a->slot < b->slot);
+}
+
+static int by_slot(const void *pa, const void *pb) {
+  int32_t a = *(const int32_t *)pa, b = *(const int32_t *)pb;
+  return (a > b) - (a < b);
+}
+
+/*
+ * Selection (Section 3.1).  n cached pairs with scores phi, budget B, the R
+ * most recent pairs protected.  Writes the kept slots in ascending order to
+ * kept[] (room for min(B, n)) and returns their number.
+ */
+int fkv_oracle_select(const float *phi, int n, int B, int R, int32_t *kept) {
+  if (n <= B) {
+    for (int i = 0; i < n; ++i) kept[i] = i;
+    return n;
+  }
+  int r = R < B ? R : B;        /* protected recent pairs */
+  int m = n - r;                /* pairs that compete */
+  int k = B - r;                /* how many of them survive */
+  ranked_t *order = (ranked_t *)malloc((size_t)(m > 0 ? m : 1) * sizeof(ranked_t));
+  for (int i = 0; i < m; ++i) { order[i].score = canonical(phi[i]); order[i].slot = i; }
+  qsort(order, (size_t)m, sizeof(ranked_t), by_score_then_slot);
+  for (int j = 0; j < k; ++j) kept[j] = order[j].slot;
+  qsort(kept, (size_t)k, sizeof(int32_t), by_slot);
+  for (int j = 0; j < r; ++j) kept[k + j] = m + j;
+  free(order);
+  return B;
+}
+
+/* Compaction (s' = s \ D): row j of the output is row kept[j] of the input. */
+void fkv_oracle_compact(const uint16_t *K, const uint16_t *V, const float *A, const int32_t *pos, int D, int F,
+                        const int32_t *kept, int nk, uint16_t *K2, uint16_t *V2, float *A2, int32_t *pos2) {
+  for (int j = 0; j < nk; ++j) {
+    size_t s = (size_t)kept[j];
+    memcpy(K2 + (size_t)j * D, K + s * D, (size_t)D * 2);
+    memcpy(V2 + (size_t)j * D, V + s * D, (size_t)D * 2);
+    memcpy(A2 + (size_t)j * F, A + s * F, (size_t)F * 4);
+    pos2[j] = pos[s];
+  }
+}
+
+/*
+ * Decode attention of the g query heads that share one KV head, over the n
+ * retained pairs (Appendix A): s_i = scale * <q, k_i>, p = softmax(s),
+ * o = sum_i p_i v_i.  q: [g][D] bf16; out_bf16: [g][D]; out_f64 (may be NULL):
+ * the same before rounding.
+ */
+void fkv_oracle_attend(const uint16_t *q, const uint16_t *K, const uint16_t *V, int n, int g, int D, double scale,
+                       uint16_t *out_bf16, double *out_f64) {
+  double *s = (double *)malloc((size_t)(n > 0 ? n : 1) * sizeof(double));
+  for (int h = 0; h < g; ++h) {
+    double mx = -INFINITY;
+    for (int i = 0; i < n; ++i) {
+      double dot = 0.0;
+      for (int c = 0; c < D; ++c) dot += bf16_to_double(q[(size_t)h * D + c]) * bf16_to_double(K[(size_t)i * D + c]);
+      s[i] = dot * scale;
+      if (s[i] > mx) mx = s[i];
+    }
+    double denom = 0.0;
+    for (int i = 0; i < n; ++i) { s[i] = exp(s[i] - mx); denom += s[i]; }
+    for (int c = 0; c < D; ++c) {
+      double acc = 0.0;
+      for (int i = 0; i < n; ++i) acc += (s[i] / denom) * bf16_to_double(V[(size_t)i * D + c]);
+      if (n == 0) acc = 0.0;
+      if (out_f64) out_f64[(size_t)h * D + c] = acc;
+      out_bf16[(size_t)h * D + c] = double_to_bf16(acc);
+    }
+  }
+  free(s);
+}
+
+/*
+ * One eviction step over many independent segments (score -> select ->
+ * compact), the unit the CPU baseline times.  Segment i has n[i] pairs laid
+ * out densely from offset off[i] (in pairs) in K, V, A, pos and phi; the
+ * outputs use the same offsets.  Scorer i is W1[i], b1[i], W2[i], b2[i].
+ * Segments run on OpenMP threads when compiled with -fopenmp; each segment is
+ * the plain sequence of the three steps above.
+ */
+void fkv_oracle_evict_batch(int nseg, const int64_t *off, const int32_t *n, const int32_t *B, int R, int D, int F,
+                            int H, int act, const uint16_t *K, const uint16_t *V, const float *A, const int32_t *pos,
+                            const float *W1, const float *b1, const float *W2, const float *b2, float *phi,
+                            int32_t *kept, int32_t *nkept, uint16_t *K2, uint16_t *V2, float *A2, int32_t *pos2) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int i = 0; i < nseg; ++i) {
+    size_t o = (size_t)off[i];
+    size_t X = (size_t)(2 * D + F);
+    fkv_oracle_score(K + o * D, V + o * D, A + o * F, n[i], D, F, H, W1 + (size_t)i * X * H, b1 + (size_t)i * H,
+                     W2 + (size_t)i * H, b2[i], act, phi + o);
+    nkept[i] = fkv_oracle_select(phi + o, n[i], B[i], R, kept + o);
+    fkv_oracle_compact(K + o * D, V + o * D, A + o * F, pos + o, D, F, kept + o, nkept[i], K2 + o * D, V2 + o * D,
+                       A2 + o * F, pos2 + o);
+  }
+}
+
+/* Decode attention over many independent segments (same threading rule). */
+void fkv_oracle_attend_batch(int nseg, const int64_t *off, const int32_t *n, int g, int D, double scale,
+                             const uint16_t *q, const uint16_t *K, const uint16_t *V, uint16_t *out) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int i = 0; i < nseg; ++i) {
+    size_t o = (size_t)off[i];
+    fkv_oracle_attend(q + (size_t)i * g * D, K + o * D, V + o * D, n[i], g, D, scale, out + (size_t)i * g * D, NULL);
+  }
+}
+
+int fkv_oracle_num_threads(void) {
+#ifdef _OPENMP
+  extern int omp_get_max_threads(void);
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}

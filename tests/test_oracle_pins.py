@@ -1,0 +1,294 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, not the oracle itself.
+
+Each part of the oracle is held against something of a different make:
+closed forms, library routines the step reduces to, brute force over tiny
+inputs, and the paper's own identity and error bound for renormalised
+attention (Appendix A).
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_03203_b200 import workloads as wl
+from util import bits, bits_to_f64, f32_to_bits, npf
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_facts.txt")
+
+
+def _facts():
+    out = {}
+    for line in open(GOLDEN):
+        line = line.split("#")[0].strip()
+        if line:
+            k, v = line.split("=", 1) if "(" not in line else line.rsplit("=", 1)
+            out[k.strip()] = float(v)
+    return out
+
+
+# ----------------------------------------------------------------- shapes the paper prints
+def test_paper_shapes_and_footprint():
+    f = _facts()
+    assert wl.FEATS_PER_HEAD == f["feats_per_head"]
+    assert wl.config(1).x_dim == f["x_dim(g=4,D=64)"]
+    assert wl.config(3).x_dim == f["x_dim(g=4,D=128)"]
+    assert wl.config(4).x_dim == f["x_dim(g=7,D=128)"]
+    w = wl.config(3)
+    assert w.scorer_hidden == f["scorer_hidden"] and wl.CHUNK == f["eviction_length"]
+    kv_bytes = w.num_layers * w.num_kv_heads * w.head_dim * 2 * 2 * w.lens[0]
+    assert abs(kv_bytes / 2 ** 30 - f["kv_bytes_qwen3_4b_32k_gib"]) < 0.01
+
+
+# ----------------------------------------------------------------- scorer
+def _rand_segment(n, D, F, H, seed):
+    rng = np.random.default_rng(seed)
+    K = f32_to_bits(rng.standard_normal((n, D)).astype(np.float32))
+    V = f32_to_bits(rng.standard_normal((n, D)).astype(np.float32))
+    A = rng.random((n, F)).astype(np.float32) * 3
+    W1 = (rng.standard_normal((2 * D + F, H)) * 0.2).astype(np.float32)
+    b1 = (rng.standard_normal(H) * 0.2).astype(np.float32)
+    W2 = rng.standard_normal(H).astype(np.float32)
+    b2 = np.float32(0.3)
+    return K, V, A, W1, b1, W2, b2
+
+
+@pytest.mark.parametrize("act,fn", [
+    (oracle.RELU, torch.relu),
+    (oracle.SILU, torch.nn.functional.silu),
+    (oracle.GELU_TANH, lambda z: torch.nn.functional.gelu(z, approximate="tanh")),
+    (oracle.SIGMOID, torch.sigmoid),
+])
+def test_score_reduces_to_two_library_matmuls(act, fn):
+    # Appendix B.1: phi = sigma(x W1 + b1) W2 + b2 is two affine maps around a pointwise
+    # function; non-square shapes (x_dim 152/29, H 16/5) catch a transposed operand.
+    for (n, D, F, H) in [(37, 64, 24, 16), (9, 8, 13, 5)]:
+        K, V, A, W1, b1, W2, b2 = _rand_segment(n, D, F, H, 1)
+        x = np.concatenate([bits_to_f64(K), bits_to_f64(V), A.astype(np.float64)], axis=1)
+        z = torch.from_numpy(x @ W1.astype(np.float64) + b1.astype(np.float64))
+        ref = (fn(z).numpy() @ W2.astype(np.float64) + float(b2)).astype(np.float32)
+        got = oracle.score(K, V, A, W1, b1, W2, b2, act)
+        np.testing.assert_allclose(got, ref, rtol=0, atol=2e-6)
+
+
+def test_score_closed_forms():
+    n, D, F, H = 11, 16, 12, 16
+    K, V, A, W1, b1, W2, b2 = _rand_segment(n, D, F, H, 2)
+    # W1 = 0: every pair scores relu(b1).W2 + b2.
+    const = float(np.maximum(b1.astype(np.float64), 0) @ W2.astype(np.float64) + b2)
+    got = oracle.score(K, V, A, np.zeros_like(W1), b1, W2, b2)
+    np.testing.assert_allclose(got, np.full(n, const, np.float32), atol=1e-7)
+    # One-hot W1 rows read back a single input channel, which fixes the order k | v | a.
+    Kf, Vf = bits_to_f64(K), bits_to_f64(V)
+    for row, column in [(3, Kf[:, 3]), (D + 5, Vf[:, 5]), (2 * D + 7, A[:, 7].astype(np.float64))]:
+        W1h = np.zeros_like(W1)
+        W1h[row, 2] = 1.0
+        W2h = np.zeros_like(W2)
+        W2h[2] = 1.0
+        got = oracle.score(K, V, A, W1h, np.zeros_like(b1), W2h, 0.0)
+        np.testing.assert_allclose(got, np.maximum(column, 0).astype(np.float32), atol=1e-7)
+    # With every pre-activation positive ReLU is the identity and phi is affine in x.
+    big = np.full_like(b1, 1e3)
+    got = oracle.score(K, V, A, W1, big, W2, b2)
+    x = np.concatenate([Kf, Vf, A.astype(np.float64)], axis=1)
+    ref = (x @ W1.astype(np.float64) + big) @ W2.astype(np.float64) + float(b2)
+    np.testing.assert_allclose(got, ref.astype(np.float32), rtol=1e-6)
+
+
+def test_score_triple_loop_brute_force():
+    n, D, F, H = 4, 3, 2, 3
+    K, V, A, W1, b1, W2, b2 = _rand_segment(n, D, F, H, 3)
+    Kf, Vf = bits_to_f64(K), bits_to_f64(V)
+    for i in range(n):
+        x = list(Kf[i]) + list(Vf[i]) + [float(a) for a in A[i]]
+        phi = float(b2)
+        for j in range(H):
+            z = float(b1[j])
+            for c in range(len(x)):
+                z += x[c] * float(W1[c][j])
+            phi += max(z, 0.0) * float(W2[j])
+        assert abs(oracle.score(K, V, A, W1, b1, W2, b2)[i] - phi) < 1e-6
+
+
+# ----------------------------------------------------------------- selection
+def _canon(s):
+    s = float(s)
+    if math.isnan(s):
+        return -math.inf
+    return 0.0 if s == 0.0 else s
+
+
+def _brute_select(phi, B, R):
+    n = len(phi)
+    if n <= B:
+        return list(range(n))
+    r = min(R, B)
+    m = n - r
+    order = sorted(range(m), key=lambda i: (-_canon(phi[i]), i))
+    return sorted(order[: B - r]) + list(range(m, n))
+
+
+def test_select_against_full_sort():
+    rng = np.random.default_rng(5)
+    for trial in range(200):
+        n = int(rng.integers(1, 80))
+        B = int(rng.integers(1, 90))
+        R = int(rng.integers(0, 20))
+        phi = rng.standard_normal(n).astype(np.float32)
+        if trial % 3 == 0:  # many exact ties
+            phi = np.round(phi * 2) / 2
+        if trial % 7 == 0:
+            phi[rng.integers(0, n)] = np.nan
+            phi[rng.integers(0, n)] = -0.0
+            phi[rng.integers(0, n)] = np.inf
+            phi[rng.integers(0, n)] = -np.inf
+        got = oracle.select(phi, B, R)
+        assert got.tolist() == _brute_select(phi, B, R), (n, B, R)
+
+
+def test_select_exhaustive_subsets_tiny():
+    # For n <= 7: among all subsets of the competing slots of the right size, the kept one
+    # is the unique subset no outsider of which beats a member under (score desc, slot asc).
+    rng = np.random.default_rng(6)
+    for n in range(2, 8):
+        for B in range(1, n):
+            for R in (0, 1, 2):
+                phi = np.round(rng.standard_normal(n) * 1.5).astype(np.float32)  # ties on purpose
+                r = min(R, B)
+                m, k = n - r, B - r
+                beats = lambda a, b: (phi[a] > phi[b]) or (phi[a] == phi[b] and a < b)
+                winners = [set(S) for S in itertools.combinations(range(m), k)
+                           if not any(beats(o, i) for i in S for o in range(m) if o not in S)]
+                assert len(winners) == 1
+                expect = sorted(winners[0]) + list(range(m, n))
+                assert oracle.select(phi, B, R).tolist() == expect
+
+
+def test_select_invariants_and_special_cases():
+    rng = np.random.default_rng(7)
+    n, B, R = 500, 200, 32
+    phi = rng.standard_normal(n).astype(np.float32)
+    kept = oracle.select(phi, B, R)
+    assert len(kept) == min(B, n)                                # Section 3.1: back to the budget
+    assert np.all(np.diff(kept) > 0)                             # ascending, no repeats
+    assert kept[-R:].tolist() == list(range(n - R, n))           # the recent window always stays
+    comp = kept[kept < n - R]
+    evicted = np.setdiff1d(np.arange(n - R), comp)
+    assert phi[evicted].max() <= phi[comp].min()                 # lowest scores are the ones evicted
+    # n <= B keeps everything; all-equal scores keep the earliest slots plus the window.
+    assert oracle.select(phi[:150], B, R).tolist() == list(range(150))
+    assert oracle.select(np.ones(n, np.float32), B, R).tolist() == list(range(B - R)) + list(range(n - R, n))
+    # R >= B keeps exactly the last B.
+    assert oracle.select(phi, 50, 80).tolist() == list(range(n - 50, n))
+    # -0 ties with +0 (lower slot wins); NaN is evicted before any number.
+    assert oracle.select(np.array([0.0, -0.0, 0.0], np.float32), 2, 0).tolist() == [0, 1]
+    assert oracle.select(np.array([np.nan, -1e30, np.nan, -np.inf], np.float32), 1, 0).tolist() == [1]
+    assert oracle.select(np.array([np.nan, np.nan, -np.inf], np.float32), 2, 0).tolist() == [0, 1]
+
+
+# ----------------------------------------------------------------- compaction
+def test_compact_rows_positions_idempotence():
+    K, V, A, W1, b1, W2, b2 = _rand_segment(300, 16, 12, 16, 8)
+    pos = np.cumsum(np.random.default_rng(8).integers(1, 5, 300)).astype(np.int32)
+    phi = oracle.score(K, V, A, W1, b1, W2, b2)
+    kept = oracle.select(phi, 100, 10)
+    K2, V2, A2, pos2 = oracle.compact(K, V, A, pos, kept)
+    assert np.array_equal(K2, K[kept]) and np.array_equal(V2, V[kept])
+    assert np.array_equal(A2, A[kept]) and np.array_equal(pos2, pos[kept])
+    assert np.all(np.diff(pos2) > 0)
+    # Evicting again at the budget changes nothing.
+    phi2 = oracle.score(K2, V2, A2, W1, b1, W2, b2)
+    np.testing.assert_array_equal(phi2, phi[kept])               # scores do not depend on the slot
+    assert oracle.select(phi2, 100, 10).tolist() == list(range(100))
+
+
+# ----------------------------------------------------------------- attention
+def test_attend_matches_library_sdpa():
+    rng = np.random.default_rng(9)
+    for (n, g, D) in [(257, 4, 64), (33, 7, 128), (1, 4, 16)]:
+        q = f32_to_bits(rng.standard_normal((g, D)).astype(np.float32))
+        K = f32_to_bits(rng.standard_normal((n, D)).astype(np.float32) * 1.5)
+        V = f32_to_bits(rng.standard_normal((n, D)).astype(np.float32))
+        tq = torch.from_numpy(bits_to_f64(q)).view(1, g, 1, D)
+        tk = torch.from_numpy(bits_to_f64(K)).view(1, 1, n, D).expand(1, g, n, D)
+        tv = torch.from_numpy(bits_to_f64(V)).view(1, 1, n, D).expand(1, g, n, D)
+        ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv).view(g, D).numpy()
+        out_b, out64 = oracle.attend(q, K, V)
+        np.testing.assert_allclose(out64, ref, atol=1e-12)
+        assert np.array_equal(out_b, f32_to_bits(ref.astype(np.float32)))
+        # an explicit scale is honoured
+        ref2 = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, scale=0.37).view(g, D).numpy()
+        np.testing.assert_allclose(oracle.attend(q, K, V, 0.37)[1], ref2, atol=1e-12)
+
+
+def test_attend_closed_forms():
+    rng = np.random.default_rng(10)
+    g, D = 4, 32
+    q = f32_to_bits(rng.standard_normal((g, D)).astype(np.float32))
+    V = f32_to_bits(rng.standard_normal((50, D)).astype(np.float32))
+    k1 = f32_to_bits(rng.standard_normal((1, D)).astype(np.float32))
+    # one retained pair: o = v_0
+    assert np.array_equal(oracle.attend(q, k1, V[:1])[0], np.broadcast_to(V[:1], (g, D)))
+    # identical keys: uniform weights, o = mean(v)
+    out64 = oracle.attend(q, np.repeat(k1, 50, axis=0), V)[1]
+    np.testing.assert_allclose(out64, np.broadcast_to(bits_to_f64(V).mean(0), (g, D)), atol=1e-13)
+
+
+def test_renormalisation_identity_and_error_bound():
+    # Appendix A: with evicted mass eps, a_hat_i = a_i / (1 - eps) on the retained set,
+    # and ||o - o_hat||_2 <= 2 C eps with C = max ||v_i||_2 - for ANY retained set.
+    rng = np.random.default_rng(11)
+    n, g, D = 400, 4, 64
+    q = f32_to_bits(rng.standard_normal((g, D)).astype(np.float32))
+    K = f32_to_bits(rng.standard_normal((n, D)).astype(np.float32))
+    V = f32_to_bits(rng.standard_normal((n, D)).astype(np.float32))
+    qf, Kf, Vf = bits_to_f64(q), bits_to_f64(K), bits_to_f64(V)
+    s = qf @ Kf.T / math.sqrt(D)
+    a = np.exp(s - s.max(1, keepdims=True))
+    a /= a.sum(1, keepdims=True)                     # full-cache attention weights
+    o_full = oracle.attend(q, K, V)[1]
+    np.testing.assert_allclose(o_full, a @ Vf, atol=1e-12)
+    C = np.linalg.norm(Vf, axis=1).max()
+    for frac in (0.9, 0.5, 0.1):
+        kept = np.sort(rng.choice(n, int(n * frac), replace=False))
+        eps = 1.0 - a[:, kept].sum(1)
+        o_hat = oracle.attend(q, K[kept], V[kept])[1]
+        np.testing.assert_allclose(o_hat, (a[:, kept] / (1 - eps)[:, None]) @ Vf[kept], atol=1e-12)
+        assert np.all(np.linalg.norm(o_full - o_hat, axis=1) <= 2 * C * eps + 1e-12)
+
+
+# ----------------------------------------------------------------- the batch drivers add nothing
+def test_batch_drivers_equal_single_segment_calls():
+    w = wl.shrink(wl.config(4), num_layers=1, max_len=300, batch=3)
+    Ks, Vs, As, Ps, ns, Bs, W1s, b1s, W2s, b2s = [], [], [], [], [], [], [], [], [], []
+    W1, b1, W2, b2 = [npf(t) for t in wl.scorer_params(w, 0)]
+    for s in range(w.batch):
+        K, V, A, pos = wl.layer_inputs(w, 0, s)
+        for h in range(w.num_kv_heads):
+            Ks.append(bits(K[h])); Vs.append(bits(V[h])); As.append(npf(A[h])); Ps.append(npf(pos))
+            ns.append(w.lens[s]); Bs.append(w.budgets[s])
+            W1s.append(W1[h]); b1s.append(b1[h]); W2s.append(W2[h]); b2s.append(b2[h])
+    off = np.concatenate([[0], np.cumsum(ns)[:-1]]).astype(np.int64)
+    phi, kept, nkept, K2, V2, A2, pos2 = oracle.evict_batch(
+        np.concatenate(Ks), np.concatenate(Vs), np.concatenate(As), np.concatenate(Ps), off, ns, Bs, 5,
+        np.stack(W1s), np.stack(b1s), np.stack(W2s), np.array(b2s))
+    q = bits(wl.queries(w, 0))
+    qs = []
+    for i in range(len(ns)):
+        p1 = oracle.score(Ks[i], Vs[i], As[i], W1s[i], b1s[i], W2s[i], b2s[i])
+        k1 = oracle.select(p1, Bs[i], 5)
+        o = int(off[i])
+        assert np.array_equal(phi[o:o + ns[i]], p1) and nkept[i] == len(k1)
+        assert np.array_equal(kept[o:o + nkept[i]], k1)
+        c = oracle.compact(Ks[i], Vs[i], As[i], Ps[i], k1)
+        assert np.array_equal(K2[o:o + nkept[i]], c[0]) and np.array_equal(pos2[o:o + nkept[i]], c[3])
+        assert np.array_equal(V2[o:o + nkept[i]], c[1]) and np.array_equal(A2[o:o + nkept[i]], c[2])
+        s, h = divmod(i, w.num_kv_heads)
+        qs.append(q[s, h * w.group_size:(h + 1) * w.group_size])
+    out = oracle.attend_batch(np.stack(qs), K2, V2, off, nkept)
+    for i in range(len(ns)):
+        o = int(off[i])
+        assert np.array_equal(out[i], oracle.attend(qs[i], K2[o:o + nkept[i]], V2[o:o + nkept[i]])[0])
