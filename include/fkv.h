@@ -1,0 +1,206 @@
+/*
+ * fkv - budgeted KV-cache eviction and decode attention for one B200 (sm_100a).
+ *
+ * C ABI of the library built from paper_2602_03203_b200/csrc.  The calls are
+ * the paper's statement of the problem (Section 3.1): a cache with budget B
+ * that grows by appended (k, v) pairs, is pruned back to B by a learned
+ * per-(layer, KV-head) scorer, and is attended over by the decode queries:
+ *
+ *     fkv_init_cache(shapes, budget)  fkv_append(k, v)  fkv_evict(layer)  fkv_decode_attn(q)
+ *
+ * Conventions
+ *   - Every function returns FKV_OK (0) or a negative fkv_status.  Nothing
+ *     throws, nothing is printed.
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are host
+ *     pointers; a pointer documented "host or dev" may be either.
+ *   - All device work is enqueued on the caller's stream (a cudaStream_t passed
+ *     as void*); calls return without synchronising unless they say "syncs".
+ *     Calls on one cache must be issued on ONE stream, or be ordered by the
+ *     caller; two calls on one cache that overlap on the GPU race.
+ *   - The library never allocates device memory for a cache.  The caller owns
+ *     one device workspace (fkv_workspace_bytes) and keeps it alive until
+ *     fkv_destroy; per-call tensors (k, v, q, out, ...) are borrowed until the
+ *     enqueued work has run.
+ *   - Device-side failures (page pool exhausted, capacity exceeded, a bounded
+ *     wait that ran out) do not fault: the kernel skips the work and sets a
+ *     bit in a status word that fkv_device_status reads.
+ *
+ * Terms: one "segment" is the cache of one (sequence, layer, KV head); it
+ * holds n "pairs" (slots 0..n-1 in position order).  D = head_dim, g =
+ * group_size (query heads per KV head), F = 6g attention features per pair
+ * (Appendix B.1), H = scorer_hidden.  bf16 tensors are passed as raw 16-bit
+ * patterns.
+ */
+#ifndef FKV_H
+#define FKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FKV_OK = 0,
+  FKV_ERR_INVALID_ARG = -1,
+  FKV_ERR_WORKSPACE_TOO_SMALL = -2,
+  FKV_ERR_CAPACITY = -3,   /* a sequence would exceed max_tokens_per_head */
+  FKV_ERR_CUDA = -4,       /* a CUDA call failed; see fkv_last_cuda_error */
+  FKV_ERR_NOT_READY = -5,  /* e.g. evict before the scorers are loaded */
+  FKV_ERR_DEVICE = -6      /* fkv_device_status found error bits */
+} fkv_status;
+
+/* Bits of the device status word (fkv_device_status). */
+#define FKV_DEV_POOL_EXHAUSTED 1u /* no free page: the step that needed it was skipped */
+#define FKV_DEV_CAPACITY 2u       /* append past max_tokens_per_head was skipped */
+#define FKV_DEV_WAIT_TIMEOUT 4u   /* a bounded wait in a kernel ran out */
+#define FKV_DEV_BAD_INDEX 8u      /* fkv_compact was given an index outside the segment */
+
+/* Scorer activation sigma.  The paper does not name it (Appendix B.1); ReLU is the default. */
+enum { FKV_ACT_RELU = 0, FKV_ACT_SILU = 1, FKV_ACT_GELU_TANH = 2, FKV_ACT_SIGMOID = 3 };
+
+#define FKV_ALL_LAYERS (-1)
+
+typedef struct fkv_cache fkv_cache; /* opaque, host side */
+
+typedef struct {
+  int32_t num_layers;
+  int32_t num_kv_heads;
+  int32_t group_size;          /* g, 1..8 */
+  int32_t head_dim;            /* D, 64 or 128 */
+  int32_t max_batch;           /* sequences */
+  int32_t page_size;           /* pairs per page; must be 16 */
+  int32_t scorer_hidden;       /* H; must be 16 (Section 4.1) */
+  int32_t activation;          /* FKV_ACT_* */
+  int32_t budget;              /* B for every sequence (fkv_set_budget overrides per sequence) */
+  int32_t recent_keep;         /* R: most recent pairs never evicted (the paper's L; 0 = plain top-B) */
+  int32_t max_tokens_per_head; /* capacity of one segment, n <= this */
+  int32_t num_pages;           /* pages in the pool; 0 = enough for every segment at capacity
+                                  plus the transient copies of an all-layer eviction */
+} fkv_config;
+
+/* Bytes of device workspace fkv_init_cache needs for this config. */
+int fkv_workspace_bytes(const fkv_config *cfg, size_t *bytes);
+
+/*
+ * init_cache(shapes, budget) - Section 3.1.  Carves the caller's device
+ * workspace (dev, 256-byte aligned, `bytes` long) into the page pool, page
+ * tables, lengths, scorer blocks and scratch, and clears it on `stream`.
+ * The handle is host memory owned by the library until fkv_destroy.
+ */
+int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, void *stream, fkv_cache **out);
+int fkv_destroy(fkv_cache *c);
+
+/* Empty every segment and return all pages to the pool (scorers and budgets stay). */
+int fkv_reset(fkv_cache *c, void *stream);
+
+/*
+ * Scorer of one (layer, KV head) - Appendix B.1:
+ *   phi = sigma(x W1 + b1) W2 + b2,  x = Concat(k, v, a).
+ * W1: host, [(2D+F)][H] row-major fp32, rows ordered k | v | a; b1, W2: host
+ * [H].  The 2D rows of W1 that multiply k and v are stored as bf16 (round to
+ * nearest even); the F feature rows, b1, W2, b2 stay fp32.  Copies to the
+ * device on `stream` from a staging buffer the handle owns (syncs).
+ */
+int fkv_load_scorer(fkv_cache *c, int layer, int kv_head, const float *W1, const float *b1, const float *W2, float b2,
+                    void *stream);
+
+/* Per-sequence budget B (host value; takes effect for later fkv_evict calls). */
+int fkv_set_budget(fkv_cache *c, int seq, int32_t budget, void *stream);
+
+/*
+ * Bulk-load one EMPTY (layer, sequence): n pairs per KV head.
+ * k, v: dev [Hkv][n][D] bf16; feat: dev [Hkv][n][F] fp32 or NULL (zeros);
+ * pos: dev [n] int32 (strictly increasing token positions) or NULL (0..n-1).
+ */
+int fkv_prefill(fkv_cache *c, int layer, int seq, const void *k, const void *v, const float *feat, const int32_t *pos,
+                int32_t n, void *stream);
+
+/*
+ * append(k, v) - Section 3.1: one new pair per sequence and KV head of `layer`.
+ * k, v: dev [max_batch][Hkv][D] bf16; pos: dev [max_batch] int32 token
+ * positions, or NULL: the position after the last stored one (0 for an empty
+ * segment).  The feature row of the new pair is zero.  seq_mask: host bitmask
+ * of the sequences that take part (bit s), 0 = all.
+ */
+int fkv_append(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, uint64_t seq_mask,
+               void *stream);
+
+/* Overwrite the feature rows of one (layer, sequence): feat dev [Hkv][n][F] fp32, n = current length. */
+int fkv_set_features(fkv_cache *c, int layer, int seq, const float *feat, void *stream);
+
+/*
+ * evict(layer) - Section 3.1 with the deterministic Top-K action: for every
+ * segment of `layer` (or of all layers, FKV_ALL_LAYERS) with n > B, score the
+ * pairs, keep the R most recent and the B - R best-scoring of the others
+ * (higher score first, then lower slot; -0 = +0, NaN lowest), and compact K, V,
+ * features and positions of the kept pairs, in position order, into fresh
+ * pages.  Afterwards n = B.  Segments with n <= B are left untouched.
+ */
+int fkv_evict(fkv_cache *c, int layer, void *stream);
+
+/*
+ * decode_attn(q) - Appendix A: out[s][h] = sum_i softmax_i(scale <q[s][h], k_i>) v_i
+ * over all retained pairs i of the KV head that query head h belongs to
+ * (h / g).  q, out: dev [max_batch][Hkv*g][D] bf16.  scale 0 means 1/sqrt(D).
+ * Sequences with n = 0 get zeros.
+ */
+int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream);
+
+/* ---- staged entry points: one kernel each, for per-step checks ---- */
+
+/* Scores of every pair of `layer`: scores_out dev [max_batch][Hkv][cap] fp32, cap = fkv_score_stride. */
+int fkv_score(fkv_cache *c, int layer, float *scores_out, void *stream);
+/*
+ * Selection from given scores (dev, same layout): writes for each segment the
+ * kept slots, ascending, to idx_out dev [max_batch][Hkv][cap] int32 and their
+ * number min(B, n) to kept_count_out dev [max_batch][Hkv].
+ */
+int fkv_select(fkv_cache *c, int layer, const float *scores_in, int32_t *idx_out, int32_t *kept_count_out,
+               void *stream);
+/*
+ * Compaction by given ascending slot lists (dev, layout as fkv_select writes
+ * them; every (sequence) must have the same count on all its heads).
+ * Syncs (reads the new lengths back).
+ */
+int fkv_compact(fkv_cache *c, int layer, const int32_t *idx, const int32_t *kept_count, void *stream);
+
+/* Row stride, in elements, of the score and index arrays above. */
+int fkv_score_stride(const fkv_cache *c, int32_t *cap);
+
+/* Dense copy of one segment: k, v dev [n][D] bf16, feat dev [n][F], pos dev [n]; any may be NULL. */
+int fkv_export_head(fkv_cache *c, int layer, int seq, int kv_head, void *k, void *v, float *feat, int32_t *pos,
+                    void *stream);
+
+/* Current lengths of `layer`: host_out [max_batch] (host mirror, no device access). */
+int fkv_get_lengths(const fkv_cache *c, int layer, int32_t *host_out);
+
+/* Reads the device status word and free-page count (syncs `stream`); clears the word. */
+int fkv_device_status(fkv_cache *c, uint32_t *status_bits, int32_t *free_pages, void *stream);
+
+/*
+ * Re-read the lengths of every layer from the device into the host mirror
+ * (syncs).  For callers that restored a saved copy of the workspace.
+ */
+int fkv_sync_lengths(fkv_cache *c, void *stream);
+
+/*
+ * Per-kernel timing of fkv_evict.  While on, fkv_evict records CUDA events on
+ * the caller's stream around its five kernels; fkv_get_evict_timing waits for
+ * the last recorded set and returns milliseconds for
+ * {plan, score, select, compact, commit}.
+ */
+int fkv_set_timing(fkv_cache *c, int on);
+int fkv_get_evict_timing(fkv_cache *c, float ms_out[5]);
+
+/* Number of kernel launches this handle has enqueued so far. */
+int fkv_launch_count(const fkv_cache *c, uint64_t *launches);
+
+/* Text of the last CUDA error seen by this library on this thread ("" if none). */
+const char *fkv_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FKV_H */

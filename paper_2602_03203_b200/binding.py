@@ -1,0 +1,232 @@
+"""Thin ctypes binding of the C ABI in ``include/fkv.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+torch is used for device memory and streams.  There is no CPU fallback: if the
+library has not been built, or no CUDA device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfkv.so")
+_lib = None
+
+ALL_LAYERS = -1
+ACT_RELU, ACT_SILU, ACT_GELU_TANH, ACT_SIGMOID = 0, 1, 2, 3
+DEV_POOL_EXHAUSTED, DEV_CAPACITY, DEV_WAIT_TIMEOUT, DEV_BAD_INDEX = 1, 2, 4, 8
+STATUS = {0: "FKV_OK", -1: "FKV_ERR_INVALID_ARG", -2: "FKV_ERR_WORKSPACE_TOO_SMALL", -3: "FKV_ERR_CAPACITY",
+          -4: "FKV_ERR_CUDA", -5: "FKV_ERR_NOT_READY", -6: "FKV_ERR_DEVICE"}
+
+EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", "fkv_load_scorer", "fkv_set_budget",
+           "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
+           "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
+           "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing"]
+
+
+class FkvConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "num_layers", "num_kv_heads", "group_size", "head_dim", "max_batch", "page_size", "scorer_hidden",
+        "activation", "budget", "recent_keep", "max_tokens_per_head", "num_pages")]
+
+
+class FkvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = f"{where}: {STATUS.get(code, code)}"
+        if code == -4:
+            msg += f" ({lib().fkv_last_cuda_error().decode()})"
+        super().__init__(msg)
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built (no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_03203_b200.build`")
+        _lib = ctypes.CDLL(LIB_PATH)
+        for name in EXPORTS:
+            getattr(_lib, name).restype = ctypes.c_int
+        _lib.fkv_last_cuda_error.restype = ctypes.c_char_p
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise FkvError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, device_type="cuda"):
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.is_contiguous() and t.device.type == device_type, (t.device, t.is_contiguous())
+    if dtype is not None:
+        assert t.dtype == dtype, (t.dtype, dtype)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Cache:
+    """One budgeted KV cache on the current CUDA device (see include/fkv.h for the semantics)."""
+
+    def __init__(self, num_layers, num_kv_heads, group_size, head_dim, max_batch, budget, max_tokens_per_head,
+                 recent_keep=0, activation=ACT_RELU, num_pages=0, page_size=16, scorer_hidden=16):
+        if not torch.cuda.is_available():
+            raise RuntimeError("fkv needs a CUDA device; there is no CPU path")
+        self.cfg = FkvConfig(num_layers, num_kv_heads, group_size, head_dim, max_batch, page_size, scorer_hidden,
+                             activation, budget, recent_keep, max_tokens_per_head, num_pages)
+        nbytes = ctypes.c_size_t(0)
+        _check(lib().fkv_workspace_bytes(ctypes.byref(self.cfg), ctypes.byref(nbytes)), "fkv_workspace_bytes")
+        self.workspace_bytes = nbytes.value
+        self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device="cuda")
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        self._h = ctypes.c_void_p(0)
+        _check(lib().fkv_init_cache(ctypes.byref(self.cfg), ctypes.c_void_p(base), ctypes.c_size_t(nbytes.value),
+                                    _stream(), ctypes.byref(self._h)), "fkv_init_cache")
+        cap = ctypes.c_int32(0)
+        _check(lib().fkv_score_stride(self._h, ctypes.byref(cap)), "fkv_score_stride")
+        self.cap = cap.value
+        self.feat_dim = 6 * group_size
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().fkv_destroy(self._h)
+            self._h = ctypes.c_void_p(0)
+            self.workspace = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- set-up
+    def reset(self):
+        _check(lib().fkv_reset(self._h, _stream()), "fkv_reset")
+
+    def load_scorer(self, layer, kv_head, W1, b1, W2, b2):
+        W1, b1, W2 = (x.detach().to("cpu", torch.float32).contiguous() for x in (W1, b1, W2))
+        _check(lib().fkv_load_scorer(self._h, layer, kv_head, _ptr(W1, torch.float32, "cpu"),
+                                     _ptr(b1, torch.float32, "cpu"), _ptr(W2, torch.float32, "cpu"),
+                                     ctypes.c_float(float(b2)), _stream()), "fkv_load_scorer")
+
+    def load_scorers(self, layer, W1, b1, W2, b2):
+        """All KV heads of a layer: W1 [Hkv][2D+F][H], b1 [Hkv][H], W2 [Hkv][H], b2 [Hkv]."""
+        W1, b1, W2, b2 = (x.detach().to("cpu", torch.float32) for x in (W1, b1, W2, b2))
+        for h in range(self.cfg.num_kv_heads):
+            self.load_scorer(layer, h, W1[h], b1[h], W2[h], float(b2[h]))
+
+    def set_budget(self, seq, budget):
+        _check(lib().fkv_set_budget(self._h, seq, int(budget), _stream()), "fkv_set_budget")
+
+    def prefill(self, layer, seq, k, v, feat=None, pos=None):
+        n = k.shape[1]
+        _check(lib().fkv_prefill(self._h, layer, seq, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
+                                 _ptr(feat, torch.float32), _ptr(pos, torch.int32), n, _stream()), "fkv_prefill")
+
+    def set_features(self, layer, seq, feat):
+        _check(lib().fkv_set_features(self._h, layer, seq, _ptr(feat, torch.float32), _stream()), "fkv_set_features")
+
+    # -- the four calls of the path
+    def append(self, layer, k, v, pos=None, seq_mask=0):
+        _check(lib().fkv_append(self._h, layer, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
+                                _ptr(pos, torch.int32), ctypes.c_uint64(seq_mask), _stream()), "fkv_append")
+
+    def evict(self, layer=ALL_LAYERS):
+        _check(lib().fkv_evict(self._h, layer, _stream()), "fkv_evict")
+
+    def decode_attn(self, layer, q, out=None, scale=0.0):
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib().fkv_decode_attn(self._h, layer, _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16),
+                                     ctypes.c_float(scale), _stream()), "fkv_decode_attn")
+        return out
+
+    # -- staged entry points
+    def score(self, layer, out=None):
+        if out is None:
+            out = torch.zeros((self.cfg.max_batch, self.cfg.num_kv_heads, self.cap), dtype=torch.float32, device="cuda")
+        _check(lib().fkv_score(self._h, layer, _ptr(out, torch.float32), _stream()), "fkv_score")
+        return out
+
+    def select(self, layer, scores):
+        idx = torch.full((self.cfg.max_batch, self.cfg.num_kv_heads, self.cap), -1, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros((self.cfg.max_batch, self.cfg.num_kv_heads), dtype=torch.int32, device="cuda")
+        _check(lib().fkv_select(self._h, layer, _ptr(scores, torch.float32), _ptr(idx, torch.int32),
+                                _ptr(cnt, torch.int32), _stream()), "fkv_select")
+        return idx, cnt
+
+    def compact(self, layer, idx, cnt):
+        _check(lib().fkv_compact(self._h, layer, _ptr(idx, torch.int32), _ptr(cnt, torch.int32), _stream()),
+               "fkv_compact")
+
+    def export_head(self, layer, seq, kv_head):
+        n = self.lengths(layer)[seq]
+        D, F = self.cfg.head_dim, self.feat_dim
+        k = torch.empty((n, D), dtype=torch.bfloat16, device="cuda")
+        v = torch.empty((n, D), dtype=torch.bfloat16, device="cuda")
+        feat = torch.empty((n, F), dtype=torch.float32, device="cuda")
+        pos = torch.empty((n,), dtype=torch.int32, device="cuda")
+        _check(lib().fkv_export_head(self._h, layer, seq, kv_head, _ptr(k), _ptr(v), _ptr(feat), _ptr(pos), _stream()),
+               "fkv_export_head")
+        return k, v, feat, pos
+
+    def lengths(self, layer):
+        arr = (ctypes.c_int32 * self.cfg.max_batch)()
+        _check(lib().fkv_get_lengths(self._h, layer, arr), "fkv_get_lengths")
+        return list(arr)
+
+    def device_status(self):
+        """(status bits, free pages); syncs the stream and clears the bits."""
+        bits, free = ctypes.c_uint32(0), ctypes.c_int32(0)
+        code = lib().fkv_device_status(self._h, ctypes.byref(bits), ctypes.byref(free), _stream())
+        if code not in (0, -6):
+            raise FkvError(code, "fkv_device_status")
+        return bits.value, free.value
+
+    def sync_lengths(self):
+        _check(lib().fkv_sync_lengths(self._h, _stream()), "fkv_sync_lengths")
+
+    def snapshot(self) -> torch.Tensor:
+        """A copy of the whole workspace (cache content, page tables, lengths, scorers)."""
+        torch.cuda.current_stream().synchronize()
+        return self.workspace.clone()
+
+    def restore(self, snap: torch.Tensor):
+        """Put a snapshot back (device-to-device copy) and refresh the host mirror of the lengths."""
+        self.workspace.copy_(snap)
+        self.sync_lengths()
+
+    def set_timing(self, on: bool):
+        _check(lib().fkv_set_timing(self._h, int(on)), "fkv_set_timing")
+
+    def evict_timing(self):
+        """Milliseconds of the last timed fkv_evict: dict plan/score/select/compact/commit."""
+        arr = (ctypes.c_float * 5)()
+        _check(lib().fkv_get_evict_timing(self._h, arr), "fkv_get_evict_timing")
+        return dict(zip(("plan", "score", "select", "compact", "commit"), (float(x) for x in arr)))
+
+    def launch_count(self):
+        n = ctypes.c_uint64(0)
+        _check(lib().fkv_launch_count(self._h, ctypes.byref(n)), "fkv_launch_count")
+        return n.value
+
+
+def from_workload(w, num_layers=None, num_pages=0, max_tokens=None) -> Cache:
+    """A cache shaped for a ``workloads.Workload`` with per-sequence budgets set."""
+    L = num_layers or w.num_layers
+    c = Cache(L, w.num_kv_heads, w.group_size, w.head_dim, w.batch, max(w.budgets),
+              max_tokens or (max(w.lens) + 256), recent_keep=w.recent_keep, activation=w.activation,
+              num_pages=num_pages)
+    for s, b in enumerate(w.budgets):
+        if b != max(w.budgets):
+            c.set_budget(s, b)
+    return c

@@ -1,0 +1,541 @@
+// Host side of the C ABI declared in include/fkv.h: argument checks, the
+// carve-up of the caller's workspace, a host mirror of the segment lengths
+// (lengths evolve deterministically, so no call reads them back), and the
+// kernel launches.  No device memory is allocated here.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/fkv.h"
+#include "fkv_attend.cuh"
+#include "fkv_aux.cuh"
+#include "fkv_compact.cuh"
+#include "fkv_dev.cuh"
+#include "fkv_score.cuh"
+#include "fkv_select.cuh"
+
+using namespace fkv;
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+constexpr int kScorePPS = 8;
+constexpr int kAttendPPS = 4;
+constexpr int kAttendStages = 3;
+constexpr int kAttendMinPages = 4;
+constexpr size_t kMaxSmem = 227 * 1024;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, part_o, part_ml,
+      tickets, total;
+  int cap, max_pages, num_pages, page_bytes, F, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
+};
+
+bool valid_config(const fkv_config *c) {
+  if (!c) return false;
+  if (c->num_layers < 1 || c->num_kv_heads < 1 || c->num_kv_heads > 32 || c->max_batch < 1 || c->max_batch > 64)
+    return false;
+  if (c->group_size < 1 || c->group_size > 8) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->page_size != kPage || c->scorer_hidden != kHidden) return false;
+  if (c->activation < 0 || c->activation > 3) return false;
+  if (c->budget < 1 || c->recent_keep < 0 || c->max_tokens_per_head < 1 || c->num_pages < 0) return false;
+  if ((int64_t)c->num_layers * c->max_batch * c->num_kv_heads > (1 << 20)) return false;
+  return true;
+}
+
+Layout make_layout(const fkv_config &c) {
+  Layout L{};
+  const int D = c.head_dim;
+  L.F = 6 * c.group_size;
+  L.cap = (int)align_up((size_t)c.max_tokens_per_head, kPage);
+  L.max_pages = L.cap / kPage;
+  L.page_bytes = 64 * D + 64 * L.F + 64;
+  const size_t nseg = (size_t)c.num_layers * c.max_batch * c.num_kv_heads;
+  const int bpages = (std::min(c.budget, L.cap) + kPage - 1) / kPage;
+  L.num_pages = c.num_pages ? c.num_pages : (int)std::min<size_t>(nseg * ((size_t)L.max_pages + bpages + 1), 0x7fffffff);
+  const int KS = 2 * D / 16;
+  L.sp_off_wf = KS * 512;
+  L.sp_off_b1 = L.sp_off_wf + L.F * 64;
+  L.sp_off_w2 = L.sp_off_b1 + 64;
+  L.sp_off_b2 = L.sp_off_w2 + 64;
+  L.sp_stride = (int)align_up((size_t)L.sp_off_b2 + 16, 256);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  L.pool = take((size_t)L.num_pages * L.page_bytes);
+  L.free_stack = take((size_t)L.num_pages * 4);
+  L.ctrl = take(CTRL_WORDS * 4);
+  L.planhdr = take(PH_WORDS * 4);
+  L.pt = take(nseg * L.max_pages * 4);
+  L.pt_new = take(nseg * L.max_pages * 4);
+  L.len = take((size_t)c.num_layers * c.max_batch * 4);
+  L.budget = take((size_t)c.max_batch * 4);
+  L.sp = take((size_t)c.num_layers * c.num_kv_heads * L.sp_stride);
+  L.scores = take(nseg * L.cap * 4);
+  L.idx = take(nseg * L.cap * 4);
+  L.plan = take(nseg * sizeof(SegPlan));
+  L.work = take(nseg * 4);
+  L.tile1 = take((nseg + 1) * 4);
+  const size_t lsegs = (size_t)c.max_batch * c.num_kv_heads;
+  L.part_o = take(lsegs * kMaxSplits * 8 * D * 4);
+  L.part_ml = take(lsegs * kMaxSplits * 8 * 2 * 4);
+  L.tickets = take(lsegs * 4);
+  L.total = off;
+  return L;
+}
+
+uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u);
+  u += 0x7fffu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+}  // namespace
+
+struct fkv_cache {
+  fkv_config cfg;
+  Layout lay;
+  Ctx ctx;
+  std::vector<int> h_len;     // [L][batch] mirror of the device lengths
+  std::vector<int> h_budget;  // [batch]
+  std::vector<uint8_t> loaded;  // [L][Hkv] scorer present
+  std::vector<uint8_t> staging;
+  uint64_t launches = 0;
+  int sm_count = 148;
+  bool timing = false, timed = false;
+  cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+};
+
+namespace {
+
+int cuda_fail(cudaError_t e) {
+  g_cuda_error = cudaGetErrorString(e);
+  return FKV_ERR_CUDA;
+}
+#define FKV_CUDA(x)                           \
+  do {                                        \
+    cudaError_t e_ = (x);                     \
+    if (e_ != cudaSuccess) return cuda_fail(e_); \
+  } while (0)
+#define FKV_LAUNCHED(c)                       \
+  do {                                        \
+    ++(c)->launches;                          \
+    cudaError_t e_ = cudaGetLastError();      \
+    if (e_ != cudaSuccess) return cuda_fail(e_); \
+  } while (0)
+
+bool layer_ok(const fkv_cache *c, int layer) { return layer >= 0 && layer < c->cfg.num_layers; }
+
+int score_stages(const fkv_cache *c) {
+  const size_t stage = (size_t)kScorePPS * ScoreSmem::pitch(c->lay.page_bytes);
+  return (int)std::max<size_t>(2, std::min<size_t>(4, (kMaxSmem - 256) / stage));
+}
+
+template <int D>
+int launch_score(fkv_cache *c, float *out, int seg_base, int tiles_bound, cudaStream_t st) {
+  const int nst = score_stages(c);
+  const size_t smem = ScoreSmem::bytes(c->lay.page_bytes, kScorePPS, nst);
+  if (smem > kMaxSmem) return FKV_ERR_INVALID_ARG;
+  static bool attr_done = false;
+  if (!attr_done) {
+    FKV_CUDA(cudaFuncSetAttribute(k_score<D, kScorePPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
+    attr_done = true;
+  }
+  const int grid = std::max(1, std::min(c->sm_count, tiles_bound));
+  k_score<D, kScorePPS><<<grid, (kScorePPS + 1) * 32, smem, st>>>(c->ctx, out, seg_base, nst);
+  FKV_LAUNCHED(c);
+  return FKV_OK;
+}
+
+int launch_score_any(fkv_cache *c, float *out, int seg_base, int tiles_bound, cudaStream_t st) {
+  return c->cfg.head_dim == 128 ? launch_score<128>(c, out, seg_base, tiles_bound, st)
+                                : launch_score<64>(c, out, seg_base, tiles_bound, st);
+}
+
+int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, int nwork_bound, cudaStream_t st) {
+  dim3 grid((max_new + kCompactRows - 1) / kCompactRows, nwork_bound);
+  if (grid.x == 0 || grid.y == 0) return FKV_OK;
+  if (c->cfg.head_dim == 128) k_compact<128><<<grid, 256, 0, st>>>(c->ctx, idx, seg_base);
+  else k_compact<64><<<grid, 256, 0, st>>>(c->ctx, idx, seg_base);
+  FKV_LAUNCHED(c);
+  return FKV_OK;
+}
+
+template <int D>
+int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale_log2, int splits, cudaStream_t st) {
+  const size_t smem = AttendSmem::bytes(D, kAttendPPS, kAttendStages);
+  static bool attr_done = false;
+  if (!attr_done) {
+    FKV_CUDA(cudaFuncSetAttribute(k_attend<D, kAttendPPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_done = true;
+  }
+  dim3 grid(splits, c->cfg.max_batch * c->cfg.num_kv_heads);
+  k_attend<D, kAttendPPS><<<grid, (kAttendPPS + 1) * 32, smem, st>>>(
+      c->ctx, layer, (const __nv_bfloat16 *)q, (__nv_bfloat16 *)out, scale_log2, kAttendMinPages, kAttendStages);
+  FKV_LAUNCHED(c);
+  return FKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int fkv_workspace_bytes(const fkv_config *cfg, size_t *bytes) {
+  if (!valid_config(cfg) || !bytes) return FKV_ERR_INVALID_ARG;
+  *bytes = make_layout(*cfg).total;
+  return FKV_OK;
+}
+
+int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, void *stream, fkv_cache **out) {
+  if (!valid_config(cfg) || !dev_workspace || !out) return FKV_ERR_INVALID_ARG;
+  if (((uintptr_t)dev_workspace & 255u) != 0) return FKV_ERR_INVALID_ARG;
+  const Layout L = make_layout(*cfg);
+  if (bytes < L.total) return FKV_ERR_WORKSPACE_TOO_SMALL;
+  fkv_cache *c = new (std::nothrow) fkv_cache();
+  if (!c) return FKV_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->lay = L;
+  uint8_t *ws = (uint8_t *)dev_workspace;
+  Ctx &x = c->ctx;
+  x.L = cfg->num_layers; x.Hkv = cfg->num_kv_heads; x.G = cfg->group_size; x.D = cfg->head_dim;
+  x.batch = cfg->max_batch; x.act = cfg->activation; x.R = cfg->recent_keep; x.F = L.F;
+  x.cap = L.cap; x.max_pages = L.max_pages; x.num_pages = L.num_pages;
+  x.page_bytes = L.page_bytes; x.off_v = 32 * cfg->head_dim; x.off_f = 64 * cfg->head_dim;
+  x.off_p = 64 * cfg->head_dim + 64 * L.F;
+  x.sp_stride = L.sp_stride; x.sp_off_wf = L.sp_off_wf; x.sp_off_b1 = L.sp_off_b1; x.sp_off_w2 = L.sp_off_w2;
+  x.sp_off_b2 = L.sp_off_b2;
+  x.pool = ws + L.pool; x.free_stack = (int *)(ws + L.free_stack); x.ctrl = (int *)(ws + L.ctrl);
+  x.planhdr = (int *)(ws + L.planhdr); x.pt = (int *)(ws + L.pt); x.pt_new = (int *)(ws + L.pt_new);
+  x.len = (int *)(ws + L.len); x.budget = (int *)(ws + L.budget); x.sp = ws + L.sp;
+  x.scores = (float *)(ws + L.scores); x.idx = (int *)(ws + L.idx); x.plan = (SegPlan *)(ws + L.plan);
+  x.work = (int *)(ws + L.work); x.tile1_start = (int *)(ws + L.tile1); x.part_o = (float *)(ws + L.part_o);
+  x.part_ml = (float *)(ws + L.part_ml); x.tickets = (int *)(ws + L.tickets);
+  c->h_len.assign((size_t)cfg->num_layers * cfg->max_batch, 0);
+  c->h_budget.assign(cfg->max_batch, cfg->budget);
+  c->loaded.assign((size_t)cfg->num_layers * cfg->num_kv_heads, 0);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  cudaStream_t st = (cudaStream_t)stream;
+  // Zero everything: freshly taken pages then hold finite values in the slots not yet written.
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws, 0, L.total, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(x.budget, c->h_budget.data(), (size_t)cfg->max_batch * 4, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    delete c;
+    return cuda_fail(e);
+  }
+  k_reset<<<256, 256, 0, st>>>(c->ctx);
+  ++c->launches;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    delete c;
+    return cuda_fail(e);
+  }
+  *out = c;
+  return FKV_OK;
+}
+
+int fkv_destroy(fkv_cache *c) {
+  if (c)
+    for (cudaEvent_t e : c->ev)
+      if (e) cudaEventDestroy(e);
+  delete c;
+  return FKV_OK;
+}
+
+int fkv_reset(fkv_cache *c, void *stream) {
+  if (!c) return FKV_ERR_INVALID_ARG;
+  k_reset<<<256, 256, 0, (cudaStream_t)stream>>>(c->ctx);
+  FKV_LAUNCHED(c);
+  std::fill(c->h_len.begin(), c->h_len.end(), 0);
+  return FKV_OK;
+}
+
+int fkv_load_scorer(fkv_cache *c, int layer, int kv_head, const float *W1, const float *b1, const float *W2, float b2,
+                    void *stream) {
+  if (!c || !layer_ok(c, layer) || kv_head < 0 || kv_head >= c->cfg.num_kv_heads || !W1 || !b1 || !W2)
+    return FKV_ERR_INVALID_ARG;
+  const int D = c->cfg.head_dim, F = c->lay.F, H = kHidden, KS = 2 * D / 16;
+  c->staging.assign(c->lay.sp_stride, 0);
+  uint32_t *wkv = (uint32_t *)c->staging.data();
+  auto w1 = [&](int row, int col) { return W1[(size_t)row * H + col]; };
+  auto pack = [&](int row, int col) {
+    return (uint32_t)f32_to_bf16_rne(w1(row, col)) | ((uint32_t)f32_to_bf16_rne(w1(row + 1, col)) << 16);
+  };
+  // mma B fragments (16 x 8, "col"): lane (gid, tig) holds rows k0 + 2 tig (+1) and k0 + 8 + 2 tig (+1) of
+  // column gid; registers 0-1 for hidden units 0-7, 2-3 for hidden units 8-15.
+  for (int ks = 0; ks < KS; ++ks)
+    for (int lane = 0; lane < 32; ++lane) {
+      const int gid = lane >> 2, tig = lane & 3, k0 = ks * 16;
+      uint32_t *r = wkv + ((size_t)ks * 32 + lane) * 4;
+      r[0] = pack(k0 + 2 * tig, gid);
+      r[1] = pack(k0 + 8 + 2 * tig, gid);
+      r[2] = pack(k0 + 2 * tig, 8 + gid);
+      r[3] = pack(k0 + 8 + 2 * tig, 8 + gid);
+    }
+  // Per quad lane t the hidden units {2t, 2t+1, 8+2t, 9+2t}: the mma accumulator columns that lane owns.
+  auto quad = [&](float *dst, auto get) {
+    for (int t = 0; t < 4; ++t) {
+      dst[t * 4 + 0] = get(2 * t); dst[t * 4 + 1] = get(2 * t + 1);
+      dst[t * 4 + 2] = get(8 + 2 * t); dst[t * 4 + 3] = get(9 + 2 * t);
+    }
+  };
+  float *wf = (float *)(c->staging.data() + c->lay.sp_off_wf);
+  for (int f = 0; f < F; ++f) quad(wf + (size_t)f * 16, [&](int j) { return w1(2 * D + f, j); });
+  quad((float *)(c->staging.data() + c->lay.sp_off_b1), [&](int j) { return b1[j]; });
+  quad((float *)(c->staging.data() + c->lay.sp_off_w2), [&](int j) { return W2[j]; });
+  *(float *)(c->staging.data() + c->lay.sp_off_b2) = b2;
+  cudaStream_t st = (cudaStream_t)stream;
+  FKV_CUDA(cudaMemcpyAsync(c->ctx.sp + ((size_t)layer * c->cfg.num_kv_heads + kv_head) * c->lay.sp_stride,
+                           c->staging.data(), c->lay.sp_stride, cudaMemcpyHostToDevice, st));
+  FKV_CUDA(cudaStreamSynchronize(st));
+  c->loaded[(size_t)layer * c->cfg.num_kv_heads + kv_head] = 1;
+  return FKV_OK;
+}
+
+int fkv_set_budget(fkv_cache *c, int seq, int32_t budget, void *stream) {
+  if (!c || seq < 0 || seq >= c->cfg.max_batch || budget < 1) return FKV_ERR_INVALID_ARG;
+  c->h_budget[seq] = budget;
+  cudaStream_t st = (cudaStream_t)stream;
+  FKV_CUDA(cudaMemcpyAsync(c->ctx.budget + seq, &c->h_budget[seq], 4, cudaMemcpyHostToDevice, st));
+  FKV_CUDA(cudaStreamSynchronize(st));
+  return FKV_OK;
+}
+
+int fkv_prefill(fkv_cache *c, int layer, int seq, const void *k, const void *v, const float *feat, const int32_t *pos,
+                int32_t n, void *stream) {
+  if (!c || !layer_ok(c, layer) || seq < 0 || seq >= c->cfg.max_batch || !k || !v || n < 1) return FKV_ERR_INVALID_ARG;
+  if (n > c->lay.cap) return FKV_ERR_CAPACITY;
+  int &hl = c->h_len[(size_t)layer * c->cfg.max_batch + seq];
+  if (hl != 0) return FKV_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  k_prefill_alloc<<<1, 1024, 0, st>>>(c->ctx, layer, seq, n);
+  FKV_LAUNCHED(c);
+  dim3 grid((n + 7) / 8, c->cfg.num_kv_heads);
+  k_prefill_rows<0><<<grid, 256, 0, st>>>(c->ctx, layer, seq, n, (const uint8_t *)k, (const uint8_t *)v, feat, pos);
+  FKV_LAUNCHED(c);
+  hl = n;
+  return FKV_OK;
+}
+
+int fkv_set_features(fkv_cache *c, int layer, int seq, const float *feat, void *stream) {
+  if (!c || !layer_ok(c, layer) || seq < 0 || seq >= c->cfg.max_batch || !feat) return FKV_ERR_INVALID_ARG;
+  const int n = c->h_len[(size_t)layer * c->cfg.max_batch + seq];
+  if (n == 0) return FKV_OK;
+  dim3 grid((n + 7) / 8, c->cfg.num_kv_heads);
+  k_prefill_rows<1><<<grid, 256, 0, (cudaStream_t)stream>>>(c->ctx, layer, seq, n, nullptr, nullptr, feat, nullptr);
+  FKV_LAUNCHED(c);
+  return FKV_OK;
+}
+
+int fkv_append(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, uint64_t seq_mask,
+               void *stream) {
+  if (!c || !layer_ok(c, layer) || !k || !v) return FKV_ERR_INVALID_ARG;
+  const int batch = c->cfg.max_batch;
+  for (int s = 0; s < batch; ++s)
+    if ((!seq_mask || ((seq_mask >> s) & 1ull)) && c->h_len[(size_t)layer * batch + s] >= c->lay.cap)
+      return FKV_ERR_CAPACITY;
+  k_append<<<batch, 32 * c->cfg.num_kv_heads, 0, (cudaStream_t)stream>>>(c->ctx, layer, (const uint8_t *)k,
+                                                                        (const uint8_t *)v, pos, seq_mask);
+  FKV_LAUNCHED(c);
+  for (int s = 0; s < batch; ++s)
+    if (!seq_mask || ((seq_mask >> s) & 1ull)) ++c->h_len[(size_t)layer * batch + s];
+  return FKV_OK;
+}
+
+int fkv_evict(fkv_cache *c, int layer, void *stream) {
+  if (!c || (layer != FKV_ALL_LAYERS && !layer_ok(c, layer))) return FKV_ERR_INVALID_ARG;
+  const int l0 = layer == FKV_ALL_LAYERS ? 0 : layer, l1 = layer == FKV_ALL_LAYERS ? c->cfg.num_layers : layer + 1;
+  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
+  int nactive = 0, max_new = 0;
+  long long tiles = 0;
+  for (int l = l0; l < l1; ++l)
+    for (int s = 0; s < batch; ++s) {
+      const int n = c->h_len[(size_t)l * batch + s], B = c->h_budget[s];
+      if (n > B) {
+        for (int h = 0; h < Hkv; ++h)
+          if (!c->loaded[(size_t)l * Hkv + h]) return FKV_ERR_NOT_READY;
+        nactive += Hkv;
+        max_new = std::max(max_new, B);
+        tiles += (long long)Hkv * ((n + kScorePPS * kPage - 1) / (kScorePPS * kPage));
+      }
+    }
+  if (nactive == 0) return FKV_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool tm = c->timing;
+  if (tm) FKV_CUDA(cudaEventRecord(c->ev[0], st));
+  k_plan<<<1, 1024, 0, st>>>(c->ctx, l0, l1, PLAN_EVICT, kScorePPS * kPage, nullptr);
+  FKV_LAUNCHED(c);
+  if (tm) FKV_CUDA(cudaEventRecord(c->ev[1], st));
+  int rc = launch_score_any(c, c->ctx.scores, 0, (int)std::min<long long>(tiles, 1 << 30), st);
+  if (rc) return rc;
+  if (tm) FKV_CUDA(cudaEventRecord(c->ev[2], st));
+  k_select<<<nactive, kSelThreads, 0, st>>>(c->ctx, c->ctx.scores, c->ctx.idx, nullptr, 0);
+  FKV_LAUNCHED(c);
+  if (tm) FKV_CUDA(cudaEventRecord(c->ev[3], st));
+  rc = launch_compact(c, c->ctx.idx, 0, max_new, nactive, st);
+  if (rc) return rc;
+  if (tm) FKV_CUDA(cudaEventRecord(c->ev[4], st));
+  k_commit<<<(l1 - l0) * batch * Hkv, 256, 0, st>>>(c->ctx, l0, l1);
+  FKV_LAUNCHED(c);
+  if (tm) {
+    FKV_CUDA(cudaEventRecord(c->ev[5], st));
+    c->timed = true;
+  }
+  for (int l = l0; l < l1; ++l)
+    for (int s = 0; s < batch; ++s) {
+      int &n = c->h_len[(size_t)l * batch + s];
+      n = std::min(n, c->h_budget[s]);
+    }
+  return FKV_OK;
+}
+
+int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream) {
+  if (!c || !layer_ok(c, layer) || !q || !out) return FKV_ERR_INVALID_ARG;
+  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads, D = c->cfg.head_dim;
+  int maxn = 0;
+  for (int s = 0; s < batch; ++s) maxn = std::max(maxn, c->h_len[(size_t)layer * batch + s]);
+  const int maxpages = (maxn + kPage - 1) / kPage;
+  int splits = (2 * c->sm_count + batch * Hkv - 1) / (batch * Hkv);
+  splits = std::max(1, std::min({splits, kMaxSplits, (maxpages + kAttendMinPages - 1) / kAttendMinPages}));
+  if (scale == 0.f) scale = 1.f / sqrtf((float)D);
+  const float scale_log2 = scale * 1.4426950408889634f;
+  cudaStream_t st = (cudaStream_t)stream;
+  return D == 128 ? launch_attend<128>(c, layer, q, out, scale_log2, splits, st)
+                  : launch_attend<64>(c, layer, q, out, scale_log2, splits, st);
+}
+
+int fkv_score_stride(const fkv_cache *c, int32_t *cap) {
+  if (!c || !cap) return FKV_ERR_INVALID_ARG;
+  *cap = c->lay.cap;
+  return FKV_OK;
+}
+
+int fkv_score(fkv_cache *c, int layer, float *scores_out, void *stream) {
+  if (!c || !layer_ok(c, layer) || !scores_out) return FKV_ERR_INVALID_ARG;
+  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
+  for (int h = 0; h < Hkv; ++h)
+    if (!c->loaded[(size_t)layer * Hkv + h]) return FKV_ERR_NOT_READY;
+  long long tiles = 0;
+  for (int s = 0; s < batch; ++s)
+    tiles += (long long)Hkv * ((c->h_len[(size_t)layer * batch + s] + kScorePPS * kPage - 1) / (kScorePPS * kPage));
+  if (tiles == 0) return FKV_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  k_plan<<<1, 1024, 0, st>>>(c->ctx, layer, layer + 1, PLAN_SCORE_ALL, kScorePPS * kPage, nullptr);
+  FKV_LAUNCHED(c);
+  return launch_score_any(c, scores_out, layer * batch * Hkv, (int)tiles, st);
+}
+
+int fkv_select(fkv_cache *c, int layer, const float *scores_in, int32_t *idx_out, int32_t *kept_count_out,
+               void *stream) {
+  if (!c || !layer_ok(c, layer) || !scores_in || !idx_out || !kept_count_out) return FKV_ERR_INVALID_ARG;
+  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
+  cudaStream_t st = (cudaStream_t)stream;
+  FKV_CUDA(cudaMemsetAsync(kept_count_out, 0, (size_t)batch * Hkv * 4, st));
+  k_plan<<<1, 1024, 0, st>>>(c->ctx, layer, layer + 1, PLAN_SELECT, kScorePPS * kPage, nullptr);
+  FKV_LAUNCHED(c);
+  k_select<<<batch * Hkv, kSelThreads, 0, st>>>(c->ctx, scores_in, idx_out, kept_count_out, layer * batch * Hkv);
+  FKV_LAUNCHED(c);
+  return FKV_OK;
+}
+
+int fkv_compact(fkv_cache *c, int layer, const int32_t *idx, const int32_t *kept_count, void *stream) {
+  if (!c || !layer_ok(c, layer) || !idx || !kept_count) return FKV_ERR_INVALID_ARG;
+  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
+  int maxn = 0;
+  for (int s = 0; s < batch; ++s) maxn = std::max(maxn, c->h_len[(size_t)layer * batch + s]);
+  if (maxn == 0) return FKV_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  k_plan<<<1, 1024, 0, st>>>(c->ctx, layer, layer + 1, PLAN_COMPACT, kScorePPS * kPage, kept_count);
+  FKV_LAUNCHED(c);
+  int rc = launch_compact(c, idx, layer * batch * Hkv, maxn, batch * Hkv, st);
+  if (rc) return rc;
+  k_commit<<<batch * Hkv, 256, 0, st>>>(c->ctx, layer, layer + 1);
+  FKV_LAUNCHED(c);
+  FKV_CUDA(cudaMemcpyAsync(&c->h_len[(size_t)layer * batch], c->ctx.len + (size_t)layer * batch, (size_t)batch * 4,
+                           cudaMemcpyDeviceToHost, st));
+  FKV_CUDA(cudaStreamSynchronize(st));
+  return FKV_OK;
+}
+
+int fkv_export_head(fkv_cache *c, int layer, int seq, int kv_head, void *k, void *v, float *feat, int32_t *pos,
+                    void *stream) {
+  if (!c || !layer_ok(c, layer) || seq < 0 || seq >= c->cfg.max_batch || kv_head < 0 || kv_head >= c->cfg.num_kv_heads)
+    return FKV_ERR_INVALID_ARG;
+  const int n = c->h_len[(size_t)layer * c->cfg.max_batch + seq];
+  if (n == 0) return FKV_OK;
+  k_export_rows<<<(n + 7) / 8, 256, 0, (cudaStream_t)stream>>>(c->ctx, layer, seq, kv_head, (uint8_t *)k, (uint8_t *)v,
+                                                               feat, pos);
+  FKV_LAUNCHED(c);
+  return FKV_OK;
+}
+
+int fkv_get_lengths(const fkv_cache *c, int layer, int32_t *host_out) {
+  if (!c || !layer_ok(c, layer) || !host_out) return FKV_ERR_INVALID_ARG;
+  for (int s = 0; s < c->cfg.max_batch; ++s) host_out[s] = c->h_len[(size_t)layer * c->cfg.max_batch + s];
+  return FKV_OK;
+}
+
+int fkv_device_status(fkv_cache *c, uint32_t *status_bits, int32_t *free_pages, void *stream) {
+  if (!c) return FKV_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int h[2] = {0, 0};
+  FKV_CUDA(cudaMemcpyAsync(h, c->ctx.ctrl, 8, cudaMemcpyDeviceToHost, st));
+  FKV_CUDA(cudaStreamSynchronize(st));
+  if (h[CTRL_STATUS]) {
+    FKV_CUDA(cudaMemsetAsync(c->ctx.ctrl + CTRL_STATUS, 0, 4, st));
+    FKV_CUDA(cudaStreamSynchronize(st));
+  }
+  if (status_bits) *status_bits = (uint32_t)h[CTRL_STATUS];
+  if (free_pages) *free_pages = h[CTRL_FREE_TOP];
+  return h[CTRL_STATUS] ? FKV_ERR_DEVICE : FKV_OK;
+}
+
+int fkv_sync_lengths(fkv_cache *c, void *stream) {
+  if (!c) return FKV_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  FKV_CUDA(cudaMemcpyAsync(c->h_len.data(), c->ctx.len, c->h_len.size() * 4, cudaMemcpyDeviceToHost, st));
+  FKV_CUDA(cudaStreamSynchronize(st));
+  return FKV_OK;
+}
+
+int fkv_set_timing(fkv_cache *c, int on) {
+  if (!c) return FKV_ERR_INVALID_ARG;
+  if (on)
+    for (cudaEvent_t &e : c->ev)
+      if (!e) FKV_CUDA(cudaEventCreate(&e));
+  c->timing = on != 0;
+  c->timed = false;
+  return FKV_OK;
+}
+
+int fkv_get_evict_timing(fkv_cache *c, float ms_out[5]) {
+  if (!c || !ms_out) return FKV_ERR_INVALID_ARG;
+  if (!c->timed) return FKV_ERR_NOT_READY;
+  FKV_CUDA(cudaEventSynchronize(c->ev[5]));
+  for (int i = 0; i < 5; ++i) FKV_CUDA(cudaEventElapsedTime(&ms_out[i], c->ev[i], c->ev[i + 1]));
+  return FKV_OK;
+}
+
+int fkv_launch_count(const fkv_cache *c, uint64_t *launches) {
+  if (!c || !launches) return FKV_ERR_INVALID_ARG;
+  *launches = c->launches;
+  return FKV_OK;
+}
+
+const char *fkv_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+}  // extern "C"

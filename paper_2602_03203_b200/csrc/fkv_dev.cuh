@@ -1,0 +1,169 @@
+// Shared device-side definitions: the cache context handed to every kernel,
+// the page-record layout, and thin wrappers over the PTX this library uses
+// (mbarrier, bulk async copy, ldmatrix, bf16 mma).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fkv {
+
+constexpr int kPage = 16;        // pairs per page
+constexpr int kHidden = 16;      // scorer hidden width (Section 4.1)
+constexpr int kMaxSplits = 64;   // split-K partials kept per segment
+
+// Device status bits (mirrors include/fkv.h).
+constexpr unsigned kDevPoolExhausted = 1u, kDevCapacity = 2u, kDevWaitTimeout = 4u, kDevBadIndex = 8u;
+
+// ctrl[] slots
+enum { CTRL_FREE_TOP = 0, CTRL_STATUS = 1, CTRL_WORDS = 8 };
+// planhdr[] slots
+enum { PH_NWORK = 0, PH_TILES1 = 1, PH_NEW_PAGES = 2, PH_OLD_PAGES = 3, PH_PUSH_START = 4, PH_WORDS = 8 };
+
+// What the plan kernel decides for one segment of the current call.
+struct SegPlan {
+  int n_old;   // pairs before
+  int n_new;   // pairs after (== n_old when the segment is left alone)
+  int r;       // protected recent pairs
+  int k_sel;   // pairs to select among slots [0, n_old - r)
+  int active;  // 1 if the segment is compacted in this call
+  int push_base;  // offset of its old pages in the push region of the free stack
+  int pad0, pad1;
+};
+
+// One page record holds 16 pairs of one segment:
+//   K   [D/64][16][64] bf16, 16-byte chunks XOR-swizzled inside each 128-byte row
+//   V   same layout
+//   a   [16][F] fp32 attention features
+//   pos [16] int32 original token positions
+// The swizzle (chunk c of row r sits at chunk c ^ (r & 7)) is the 128-byte
+// shared-memory swizzle, applied in HBM so that ONE bulk copy of the record
+// lands in shared memory ready for conflict-free ldmatrix.
+struct Ctx {
+  int L, Hkv, G, D, batch, act, R, F;
+  int cap;        // segment capacity in pairs (multiple of 16)
+  int max_pages;  // cap / 16
+  int num_pages;
+  int page_bytes, off_v, off_f, off_p;
+  int sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
+  uint8_t *pool;
+  int *free_stack;
+  int *ctrl;
+  int *pt, *pt_new;  // [L][batch][Hkv][max_pages]
+  int *len;          // [L][batch]
+  int *budget;       // [batch]
+  uint8_t *sp;       // scorer blocks [L][Hkv]
+  float *scores;     // [L][batch][Hkv][cap]
+  int *idx;          // [L][batch][Hkv][cap]
+  SegPlan *plan;     // [L*batch*Hkv]
+  int *work;         // work list of segment ids
+  int *tile1_start;  // prefix of score tiles over the work list
+  int *planhdr;
+  float *part_o;     // [batch*Hkv][kMaxSplits][8][D]
+  float *part_ml;    // [batch*Hkv][kMaxSplits][8][2]
+  int *tickets;      // [batch*Hkv]
+};
+
+__device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head) {
+  return (layer * c.batch + seq) * c.Hkv + head;
+}
+
+// Byte offset, inside the K (or V) part of a page record, of 16-byte chunk `ch`
+// (8 channels) of row `r`.
+__device__ __forceinline__ int kv_chunk_off(int r, int ch) {
+  return ((ch >> 3) << 11) + (r << 7) + (((ch & 7) ^ (r & 7)) << 4);
+}
+
+__device__ __forceinline__ void set_status(const Ctx &c, unsigned bits) { atomicOr((unsigned *)&c.ctrl[CTRL_STATUS], bits); }
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+// Bounded wait on a phase parity.  try_wait suspends for a hardware time slice
+// per call, so the cap is seconds, far beyond any copy latency; false = gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < (1u << 22); ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// One-dimensional bulk copy global -> shared, completion counted in bytes on an mbarrier.
+// Both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Block-wide exclusive prefix sum of one int per thread (blockDim.x <= 1024,
+// a multiple of 32).  `total` gets the block total.  smem: 33 ints.
+__device__ __forceinline__ int block_excl_scan(int v, int *smem, int &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();  // smem may still be read from a previous call
+  if (lane == 31) smem[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = lane < nw ? smem[lane] : 0, winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    smem[lane] = winc - w;
+    if (lane == 31) smem[32] = winc;
+  }
+  __syncthreads();
+  total = smem[32];
+  return smem[warp] + inc - v;
+}
+
+}  // namespace fkv
