@@ -1,0 +1,332 @@
+#!/usr/bin/env python
+"""Benchmark of the eviction + decode-attention hot path on B200.
+
+A step is one pass of the whole hot path over one batch of synthetic input:
+one budgeted eviction over all layers (score -> select -> compact), then T
+decode tokens (append + GQA decode attention in every layer).  The cache is
+put back to its pre-eviction content between steps (untimed), and an L2-sized
+buffer is overwritten so every step starts cold.
+
+Prints ONE JSON line.  `value` is the eviction step's algorithmic HBM
+throughput (GB/s); decode tokens/s, per-kernel times, the roofline of the
+dominant kernel and the CPU oracle's timing ride along.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--config 1..5] [--budget B] [--decode-tokens T]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2602_03203_b200 import workloads as wl
+
+METRIC = "eviction_step_hbm_throughput"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0      # the "~8 TB/s" the target is quoted against
+FALLBACK_HBM_GBS = 6650.0     # used only when MEASURED_PEAKS.json is absent
+
+
+# ----------------------------------------------------------------------------- algorithmic bytes
+def pair_bytes(w):
+    return 4 * w.head_dim + 4 * w.feat_dim + 4      # K + V rows (bf16), feature row (fp32), position id
+
+
+def evict_bytes(w, num_layers):
+    """Algorithmic HBM bytes of one eviction: per pair, the scorer reads K, V, features and
+    writes a 4-byte score; selection reads the score and writes 4 bytes per kept pair;
+    compaction reads and writes K, V, features and position of every kept pair plus its index."""
+    score = select = compact = 0
+    for n, B in zip(w.lens, w.budgets):
+        if n <= B:
+            continue
+        segs = num_layers * w.num_kv_heads
+        score += segs * n * (pair_bytes(w) - 4 + 4)
+        select += segs * (4 * n + 4 * B)
+        compact += segs * B * (2 * pair_bytes(w) + 4)
+    return dict(score=score, select=select, compact=compact, total=score + select + compact)
+
+
+def decode_bytes_per_token(w, num_layers, lens_now):
+    return sum(num_layers * w.num_kv_heads * n * 4 * w.head_dim for n in lens_now)
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0])); mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for nm, val in zip(names, parts[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(nm)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(w, target_s=12.0, max_layers=4):
+    """Times the oracle's eviction step (score -> select -> compact) on whole layers of the
+    workload until about `target_s` seconds of CPU work are done."""
+    import oracle
+    from paper_2602_03203_b200.workloads import layer_inputs, scorer_params
+    threads = oracle.num_threads()
+    spent, bytes_done, pairs_done, layers_done = 0.0, 0, 0, 0
+    for l in range(min(max_layers, w.num_layers)):
+        Ks, Vs, As, Ps, ns, Bs, W1s, b1s, W2s, b2s = [], [], [], [], [], [], [], [], [], []
+        W1, b1, W2, b2 = [t.numpy() for t in scorer_params(w, l)]
+        for s in range(w.batch):
+            K, V, A, pos = layer_inputs(w, l, s)
+            Kb = K.view(torch.int16).numpy().view(np.uint16)
+            Vb = V.view(torch.int16).numpy().view(np.uint16)
+            for h in range(w.num_kv_heads):
+                Ks.append(Kb[h]); Vs.append(Vb[h]); As.append(A[h].numpy()); Ps.append(pos.numpy())
+                ns.append(w.lens[s]); Bs.append(w.budgets[s])
+                W1s.append(W1[h]); b1s.append(b1[h]); W2s.append(W2[h]); b2s.append(b2[h])
+        off = np.concatenate([[0], np.cumsum(ns)[:-1]]).astype(np.int64)
+        args = (np.concatenate(Ks), np.concatenate(Vs), np.concatenate(As), np.concatenate(Ps), off, ns, Bs,
+                w.recent_keep, np.stack(W1s), np.stack(b1s), np.stack(W2s), np.array(b2s), w.activation)
+        t0 = time.perf_counter()
+        oracle.evict_batch(*args)
+        dt = time.perf_counter() - t0
+        spent += dt
+        layers_done += 1
+        bytes_done += evict_bytes(w, 1)["total"]
+        pairs_done += sum(ns)
+        if spent >= target_s:
+            break
+    return dict(seconds=spent, bytes=bytes_done, pairs=pairs_done, layers=layers_done, threads=threads)
+
+
+def run_reference(args):
+    """The reference arm: there is no reference implementation, so the CPU oracle, as it
+    stands, is timed on the host cores on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.config(args.config, budget=args.budget)
+    per_step = []
+    sample = None
+    for i in range(args.warmup + args.steps):
+        sample = oracle_sample(w, target_s=0.0, max_layers=1)      # one layer per step
+        if i >= args.warmup:
+            per_step.append(sample["seconds"])
+    ms = 1e3 * sum(per_step) / max(1, len(per_step))
+    gbs = sample["bytes"] / (ms * 1e-3) / 1e9
+    desc = f"layer 0 of {w.num_layers} ({sample['pairs']} pairs) per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "budget": w.budgets[0], "sample": desc},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": sample["threads"], "kind": "oracle", "sample": desc},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+def run_ours(args):
+    from paper_2602_03203_b200 import binding
+    from paper_2602_03203_b200.dist import Ranks
+
+    ranks = Ranks()                      # one process per GPU; no collective on the data path
+    torch.cuda.set_device(ranks.local_rank)
+    dev = torch.device("cuda", ranks.local_rank)
+    w = wl.config(args.config, budget=args.budget)
+    L = args.layers or w.num_layers
+    T = args.decode_tokens
+    cache = binding.from_workload(w, L, max_tokens=max(w.lens) + max(256, T))
+    for l in range(L):
+        cache.load_scorers(l, *wl.scorer_params(w, l, dev))
+        for s in range(w.batch):
+            K, V, A, pos = wl.layer_inputs(w, l, s, dev)
+            cache.prefill(l, s, K, V, A, pos)
+            del K, V, A, pos
+    torch.cuda.synchronize()
+    snap = cache.snapshot()
+    status, _ = cache.device_status()
+    assert status == 0, f"device status {status} after prefill"
+
+    # Decode inputs of one step, resident (device arm) and in pinned host memory (end-to-end arm).
+    g0 = torch.Generator(device=dev); g0.manual_seed(1234 + w.seed)
+    kd = torch.randn((T, L, w.batch, w.num_kv_heads, w.head_dim), generator=g0, device=dev).to(torch.bfloat16)
+    vd = torch.randn((T, L, w.batch, w.num_kv_heads, w.head_dim), generator=g0, device=dev).to(torch.bfloat16)
+    qd = torch.randn((T, L, w.batch, w.num_q_heads, w.head_dim), generator=g0, device=dev).to(torch.bfloat16)
+    od = torch.empty_like(qd)
+    kh, vh, qh = (x.cpu().pin_memory() for x in (kd, vd, qd))
+    oh = torch.empty(od.shape, dtype=od.dtype).pin_memory()
+    kept_dev = torch.empty((L, w.batch, w.num_kv_heads, max(w.budgets)), dtype=torch.int32, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)        # > 126 MB of L2
+
+    eb = evict_bytes(w, L)
+    lens_after = [min(n, b) for n, b in zip(w.lens, w.budgets)]
+    dec_bytes = sum(decode_bytes_per_token(w, L, [n + t + 1 for n in lens_after]) for t in range(T))
+    cache.set_timing(True)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+
+    def one_step(e2e: bool):
+        cache.restore(snap)
+        flush.fill_(1)
+        torch.cuda.synchronize()
+        ev[0].record()
+        if e2e:
+            kd.copy_(kh, non_blocking=True); vd.copy_(vh, non_blocking=True); qd.copy_(qh, non_blocking=True)
+        ev[1].record()
+        cache.evict(binding.ALL_LAYERS)
+        ev[2].record()
+        for t in range(T):
+            cache.decode_step(kd[t], vd[t], qd[t], od[t])
+        if e2e:
+            oh.copy_(od, non_blocking=True)
+        ev[3].record()
+        torch.cuda.synchronize()
+        return dict(h2d=ev[0].elapsed_time(ev[1]), evict=ev[1].elapsed_time(ev[2]), decode=ev[2].elapsed_time(ev[3]),
+                    kernels=cache.evict_timing())
+
+    for _ in range(args.warmup):
+        one_step(False)
+    ranks.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(ranks.local_rank)
+    sampler.start()
+    launches0 = cache.launch_count()
+    res = [one_step(False) for _ in range(args.steps)]
+    launches = cache.launch_count() - launches0
+    torch.cuda.synchronize()
+    ranks.barrier()
+    clocks = sampler.stop()
+    e2e_res = [one_step(True) for _ in range(max(1, min(args.steps, 3)))]
+    status, _ = cache.device_status()
+    assert status == 0, f"device status {status}"
+
+    mean = lambda xs: sum(xs) / len(xs)
+    evict_ms = ranks.max(mean([r["evict"] for r in res]))
+    decode_ms = ranks.max(mean([r["decode"] for r in res]))
+    kern = {k: ranks.max(mean([r["kernels"][k] for r in res])) for k in res[0]["kernels"]}
+    N = ranks.world
+    value = N * eb["total"] / (evict_ms * 1e-3) / 1e9
+    tok_s = N * w.batch * T / (decode_ms * 1e-3) if T else 0.0
+    e_evict = ranks.max(mean([r["h2d"] + r["evict"] for r in e2e_res]))
+    e_decode = ranks.max(mean([r["decode"] for r in e2e_res]))
+    peak, peak_kind = measured_peak()
+    dom = "score" if kern["score"] >= kern["compact"] else "compact"
+    dom_bytes = eb[dom]
+    achieved = dom_bytes / (kern[dom] * 1e-3) / 1e9
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": N, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": evict_ms + decode_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "layers": L, "kv_heads": w.num_kv_heads, "group_size": w.group_size,
+                   "head_dim": w.head_dim, "batch": w.batch, "context": max(w.lens), "budget": max(w.budgets),
+                   "recent_keep": w.recent_keep, "decode_tokens_per_step": T, "parallelism": f"replicas{N}",
+                   "l2": "cache restored and a 512 MiB buffer overwritten before every step; inputs exceed L2"},
+        "evict_ms": evict_ms, "decode_ms": decode_ms, "kernel_ms": kern,
+        "evict_bytes": eb, "evict_frac_of_measured_peak": value / N / peak,
+        "evict_frac_of_nominal_8TBps": value / N / NOMINAL_HBM_GBS,
+        "decode_tokens_per_s": tok_s,
+        "decode_attn_gbs": N * dec_bytes / (decode_ms * 1e-3) / 1e9 if T else 0.0,
+        "roofline": {"bound": "hbm", "kernel": f"k_{dom}", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": args.traffic},
+        "e2e": {"value": N * eb["total"] / (e_evict * 1e-3) / 1e9, "unit": UNIT,
+                "decode_tokens_per_s": N * w.batch * T / (e_decode * 1e-3) if T else 0.0,
+                "h2d_bytes_per_step": kh.numel() * 2 + vh.numel() * 2 + qh.numel() * 2,
+                "d2h_bytes_per_step": oh.numel() * 2,
+                "note": "pinned-host decode inputs copied in before the eviction, attention outputs copied out"},
+        "gpu_launches": launches, "clocks": clocks,
+    }
+    if ranks.rank == 0 and N == 1 and not args.no_cpu_baseline:
+        smp = oracle_sample(w)
+        line["cpu_baseline"] = {
+            "value": smp["bytes"] / smp["seconds"] / 1e9, "unit": UNIT, "cores": smp["threads"], "kind": "oracle",
+            "sample": f"{smp['layers']} of {w.num_layers} layers ({smp['pairs']} pairs), score+select+compact, "
+                      f"{smp['seconds']:.1f} s"}
+    if ranks.rank == 0:
+        print(json.dumps(line))
+    ranks.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=3)
+    ap.add_argument("--budget", type=int, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="fewer layers (profiling captures only)")
+    ap.add_argument("--decode-tokens", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per launch of the dominant kernel")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

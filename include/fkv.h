@@ -148,6 +148,17 @@ int fkv_evict(fkv_cache *c, int layer, void *stream);
  */
 int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream);
 
+/*
+ * One decode token through every layer, in layer order: for l = 0 .. L-1,
+ * append(k[l], v[l]) then decode_attn(q[l]) -> out[l].  k, v: dev
+ * [L][max_batch][Hkv][D] bf16; q, out: dev [L][max_batch][Hkv*g][D] bf16; pos:
+ * dev [max_batch] or NULL (as fkv_append).  Exactly the two calls above issued
+ * L times from native code (a driver loop for engines that have all layers'
+ * tensors at hand, and for benchmarks of the attention side alone).
+ */
+int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *pos, const void *q, void *out,
+                    float scale, void *stream);
+
 /* ---- staged entry points: one kernel each, for per-step checks ---- */
 
 /* Scores of every pair of `layer`: scores_out dev [max_batch][Hkv][cap] fp32, cap = fkv_score_stride. */

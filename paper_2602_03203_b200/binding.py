@@ -25,7 +25,8 @@ STATUS = {0: "FKV_OK", -1: "FKV_ERR_INVALID_ARG", -2: "FKV_ERR_WORKSPACE_TOO_SMA
 EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", "fkv_load_scorer", "fkv_set_budget",
            "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
            "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
-           "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing"]
+           "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing",
+           "fkv_decode_step"]
 
 
 class FkvConfig(ctypes.Structure):
@@ -148,6 +149,15 @@ class Cache:
             out = torch.empty_like(q)
         _check(lib().fkv_decode_attn(self._h, layer, _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16),
                                      ctypes.c_float(scale), _stream()), "fkv_decode_attn")
+        return out
+
+    def decode_step(self, k, v, q, out=None, pos=None, scale=0.0):
+        """One token through all layers: k, v [L][batch][Hkv][D]; q, out [L][batch][Hq][D]."""
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib().fkv_decode_step(self._h, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16), _ptr(pos, torch.int32),
+                                     _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16), ctypes.c_float(scale),
+                                     _stream()), "fkv_decode_step")
         return out
 
     # -- staged entry points

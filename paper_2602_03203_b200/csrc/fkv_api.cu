@@ -418,6 +418,20 @@ int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float sca
                   : launch_attend<64>(c, layer, q, out, scale_log2, splits, st);
 }
 
+int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *pos, const void *q, void *out,
+                    float scale, void *stream) {
+  if (!c || !k || !v || !q || !out) return FKV_ERR_INVALID_ARG;
+  const size_t kv_stride = (size_t)c->cfg.max_batch * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
+  const size_t q_stride = kv_stride * c->cfg.group_size;
+  for (int l = 0; l < c->cfg.num_layers; ++l) {
+    int rc = fkv_append(c, l, (const uint8_t *)k + l * kv_stride, (const uint8_t *)v + l * kv_stride, pos, 0, stream);
+    if (rc) return rc;
+    rc = fkv_decode_attn(c, l, (const uint8_t *)q + l * q_stride, (uint8_t *)out + l * q_stride, scale, stream);
+    if (rc) return rc;
+  }
+  return FKV_OK;
+}
+
 int fkv_score_stride(const fkv_cache *c, int32_t *cap) {
   if (!c || !cap) return FKV_ERR_INVALID_ARG;
   *cap = c->lay.cap;

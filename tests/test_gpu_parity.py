@@ -250,9 +250,12 @@ def _attn_check(ld, layer, step=0):
     for s in range(w.batch):
         for h in range(w.num_kv_heads):
             k2, v2, _, _ = ld.export(layer, s, h)
-            ref, _ = oracle.attend(qb[s, h * g:(h + 1) * g], k2, v2)
-            err = np.abs(bits_to_f64(out_b[s, h * g:(h + 1) * g]) - bits_to_f64(ref)).max()
-            worst = max(worst, float(err))
+            ref, ref64 = oracle.attend(qb[s, h * g:(h + 1) * g], k2, v2)
+            err = np.abs(bits_to_f64(out_b[s, h * g:(h + 1) * g]) - bits_to_f64(ref))
+            # 2e-2 absolute; where one bf16 step is coarser than that (|o| >= 2.56) one step is allowed,
+            # since two correctly rounded results can land on neighbouring bf16 values.
+            allowed = np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64))
+            worst = max(worst, float((err / allowed).max()) * ATTN_TOL)
     return worst
 
 
