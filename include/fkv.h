@@ -208,6 +208,42 @@ int fkv_get_evict_timing(fkv_cache *c, float ms_out[5]);
 /* Number of kernel launches this handle has enqueued so far. */
 int fkv_launch_count(const fkv_cache *c, uint64_t *launches);
 
+/*
+ * Decode attention without any allocation (the paper has no counterpart; this
+ * is a service entry point of the library).
+ *
+ * For callers that may not allocate device memory: code running inside a
+ * memory pool that was sized once and frozen, a serving process that accounts
+ * for every byte of HBM itself, a plug-in that is handed tensors and nothing
+ * else.  Such a caller cannot provide the workspace fkv_init_cache needs, so
+ * this call takes dense tensors and keeps its split-K partials in a fixed
+ * array inside the library image (about 1.1 MB of HBM on every GPU that loads
+ * the library, held until the process exits).  It calls no cudaMalloc,
+ * cudaFree or other allocating routine.
+ *
+ *   out[h] = sum_i softmax_i(scale <q[h], k[h / g][i]>) v[h / g][i],  i < n
+ *
+ * q, out: dev [num_kv_heads * group_size][head_dim] bf16; k, v: dev
+ * [num_kv_heads][n][head_dim] bf16, dense row-major; scale 0 means
+ * 1/sqrt(head_dim).  Same arithmetic as fkv_decode_attn (fp32 online softmax,
+ * bf16 result), for one sequence.
+ *
+ * Limits: head_dim 64 or 128 (else FKV_ERR_INVALID_ARG); 1 <= n <=
+ * FKV_NOALLOC_MAX_PAIRS, num_kv_heads <= FKV_NOALLOC_MAX_KV_HEADS, group_size
+ * <= 8 - beyond them the call does nothing and returns FKV_ERR_CAPACITY.
+ *
+ * The first call on a device looks up the array's device address (once per
+ * device, with that device current); make that first call before any stream
+ * capture begins.  All calls share the one array, which keeps the previous
+ * call's partials (the call clears the only part that must start at zero):
+ * two calls that overlap on the GPU - different streams, or different
+ * threads without ordering - race on it.  Order them on one stream.
+ */
+#define FKV_NOALLOC_MAX_PAIRS (1 << 20)
+#define FKV_NOALLOC_MAX_KV_HEADS 16
+int fkv_decode_attn_dense_noalloc(const void *q, const void *k, const void *v, int32_t n, int32_t num_kv_heads,
+                                  int32_t group_size, int32_t head_dim, float scale, void *out, void *stream);
+
 /* Text of the last CUDA error seen by this library on this thread ("" if none). */
 const char *fkv_last_cuda_error(void);
 

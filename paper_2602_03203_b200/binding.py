@@ -26,7 +26,7 @@ EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", 
            "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
            "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
            "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing",
-           "fkv_decode_step"]
+           "fkv_decode_step", "fkv_decode_attn_dense_noalloc"]
 
 
 class FkvConfig(ctypes.Structure):
@@ -228,6 +228,24 @@ class Cache:
         n = ctypes.c_uint64(0)
         _check(lib().fkv_launch_count(self._h, ctypes.byref(n)), "fkv_launch_count")
         return n.value
+
+
+def decode_attn_dense_noalloc(q, k, v, group_size, out=None, scale=0.0):
+    """Decode attention over dense K/V with no allocation inside the library.
+
+    For callers that cannot give the library a workspace (a frozen memory pool, a host
+    process that owns all of HBM): q [Hkv*g][D], k, v [Hkv][n][D], all bf16 on the device.
+    The split-K partials sit in a fixed array inside the library; calls must not overlap
+    on the GPU.  Returns out [Hkv*g][D] (pass `out` to avoid torch allocating it).
+    """
+    Hkv, n, D = k.shape
+    if out is None:
+        out = torch.empty_like(q)
+    code = lib().fkv_decode_attn_dense_noalloc(_ptr(q, torch.bfloat16), _ptr(k, torch.bfloat16),
+                                               _ptr(v, torch.bfloat16), n, Hkv, group_size, D, ctypes.c_float(scale),
+                                               _ptr(out, torch.bfloat16), _stream())
+    _check(code, "fkv_decode_attn_dense_noalloc")
+    return out
 
 
 def from_workload(w, num_layers=None, num_pages=0, max_tokens=None) -> Cache:
