@@ -125,7 +125,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample(w, target_s=12.0, max_layers=4):
+def oracle_sample(w, target_s=10.0, max_layers=64):
     """Times the oracle's eviction step (score -> select -> compact) on whole layers of the
     workload until about `target_s` seconds of CPU work are done."""
     import oracle

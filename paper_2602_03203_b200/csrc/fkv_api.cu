@@ -360,7 +360,7 @@ int fkv_evict(fkv_cache *c, int layer, void *stream) {
   if (!c || (layer != FKV_ALL_LAYERS && !layer_ok(c, layer))) return FKV_ERR_INVALID_ARG;
   const int l0 = layer == FKV_ALL_LAYERS ? 0 : layer, l1 = layer == FKV_ALL_LAYERS ? c->cfg.num_layers : layer + 1;
   const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
-  int nactive = 0, max_new = 0;
+  int nactive = 0, max_new = 0, max_old = 0;
   long long tiles = 0;
   for (int l = l0; l < l1; ++l)
     for (int s = 0; s < batch; ++s) {
@@ -370,6 +370,7 @@ int fkv_evict(fkv_cache *c, int layer, void *stream) {
           if (!c->loaded[(size_t)l * Hkv + h]) return FKV_ERR_NOT_READY;
         nactive += Hkv;
         max_new = std::max(max_new, B);
+        max_old = std::max(max_old, n);
         tiles += (long long)Hkv * ((n + kScorePPS * kPage - 1) / (kScorePPS * kPage));
       }
     }
@@ -383,7 +384,8 @@ int fkv_evict(fkv_cache *c, int layer, void *stream) {
   int rc = launch_score_any(c, c->ctx.scores, 0, (int)std::min<long long>(tiles, 1 << 30), st);
   if (rc) return rc;
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[2], st));
-  k_select<<<nactive, kSelThreads, 0, st>>>(c->ctx, c->ctx.scores, c->ctx.idx, nullptr, 0);
+  if (max_old <= kSelRound) k_select<true><<<nactive, kSelThreads, 0, st>>>(c->ctx, c->ctx.scores, c->ctx.idx, nullptr, 0, 1);
+  else k_select<false><<<nactive, kSelThreads, 0, st>>>(c->ctx, c->ctx.scores, c->ctx.idx, nullptr, 0, 1);
   FKV_LAUNCHED(c);
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[3], st));
   rc = launch_compact(c, c->ctx.idx, 0, max_new, nactive, st);
@@ -461,7 +463,12 @@ int fkv_select(fkv_cache *c, int layer, const float *scores_in, int32_t *idx_out
   FKV_CUDA(cudaMemsetAsync(kept_count_out, 0, (size_t)batch * Hkv * 4, st));
   k_plan<<<1, 1024, 0, st>>>(c->ctx, layer, layer + 1, PLAN_SELECT, kScorePPS * kPage, nullptr);
   FKV_LAUNCHED(c);
-  k_select<<<batch * Hkv, kSelThreads, 0, st>>>(c->ctx, scores_in, idx_out, kept_count_out, layer * batch * Hkv);
+  int max_old = 0;
+  for (int s = 0; s < batch; ++s) max_old = std::max(max_old, c->h_len[(size_t)layer * batch + s]);
+  if (max_old <= kSelRound)
+    k_select<true><<<batch * Hkv, kSelThreads, 0, st>>>(c->ctx, scores_in, idx_out, kept_count_out, layer * batch * Hkv, 0);
+  else
+    k_select<false><<<batch * Hkv, kSelThreads, 0, st>>>(c->ctx, scores_in, idx_out, kept_count_out, layer * batch * Hkv, 0);
   FKV_LAUNCHED(c);
   return FKV_OK;
 }
@@ -474,6 +481,8 @@ int fkv_compact(fkv_cache *c, int layer, const int32_t *idx, const int32_t *kept
   if (maxn == 0) return FKV_OK;
   cudaStream_t st = (cudaStream_t)stream;
   k_plan<<<1, 1024, 0, st>>>(c->ctx, layer, layer + 1, PLAN_COMPACT, kScorePPS * kPage, kept_count);
+  FKV_LAUNCHED(c);
+  k_fill_pt_new<<<batch * Hkv, 256, 0, st>>>(c->ctx, layer * batch * Hkv, batch * Hkv);
   FKV_LAUNCHED(c);
   int rc = launch_compact(c, idx, layer * batch * Hkv, maxn, batch * Hkv, st);
   if (rc) return rc;

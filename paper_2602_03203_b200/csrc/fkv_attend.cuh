@@ -205,19 +205,57 @@ __global__ void __launch_bounds__((PPS + 1) * 32) k_attend(Ctx c, int layer, con
   __syncthreads();
   if (!s_last) return;
   __threadfence();
+  // Weights of the splits per query row: w[r][s] = 2^(m_s - M_r) / sum_s 2^(m_s - M_r) l_s, in shared memory.
+  float *s_w = reinterpret_cast<float *>(smem);  // [8][kMaxSplits] m then weights; [8][kMaxSplits] l; ring is idle
+  float *s_l = s_w + 8 * kMaxSplits;
   const float *ao = c.part_o + (size_t)y * kMaxSplits * 8 * D;
-  const float *aml = c.part_ml + (size_t)y * kMaxSplits * 8 * 2;
-  for (int e = tid; e < G * D; e += blockDim.x) {
-    const int r = e / D, ch = e - r * D;
+  const float2 *aml = reinterpret_cast<const float2 *>(c.part_ml + (size_t)y * kMaxSplits * 8 * 2);
+  __syncthreads();
+  for (int e = tid; e < G * ns; e += blockDim.x) {
+    const int r = e / ns, sidx = e - r * ns;
+    const float2 ml = __ldcg(aml + sidx * 8 + r);
+    s_w[r * kMaxSplits + sidx] = ml.x;
+    s_l[r * kMaxSplits + sidx] = ml.y;
+  }
+  __syncthreads();
+  for (int r = warp; r < G; r += PPS + 1) {  // one warp per query row
+    float *w = s_w + r * kMaxSplits, *l = s_l + r * kMaxSplits;
     float M = -INFINITY;
-    for (int sidx = 0; sidx < ns; ++sidx) M = fmaxf(M, __ldcg(aml + (sidx * 8 + r) * 2));
-    float acc = 0.f, l = 0.f;
-    for (int sidx = 0; sidx < ns; ++sidx) {
-      const float f = exp2f(__ldcg(aml + (sidx * 8 + r) * 2) - M);
-      acc += f * __ldcg(ao + ((size_t)sidx * 8 + r) * D + ch);
-      l += f * __ldcg(aml + (sidx * 8 + r) * 2 + 1);
+    for (int sidx = lane; sidx < ns; sidx += 32) M = fmaxf(M, w[sidx]);
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o2));
+    float L = 0.f;
+    for (int sidx = lane; sidx < ns; sidx += 32) {
+      const float f = exp2f(w[sidx] - M);
+      w[sidx] = f;
+      L += f * l[sidx];
     }
-    out[(qrow0 + r) * D + ch] = __float2bfloat16(acc / l);
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o2);
+    const float inv = 1.f / L;
+    for (int sidx = lane; sidx < ns; sidx += 32) w[sidx] *= inv;
+  }
+  __syncthreads();
+  // Each thread owns 4 consecutive channels of one query row; the loads of 8 splits are in flight together.
+  for (int e = tid; e < G * (D / 4); e += blockDim.x) {
+    const int r = e / (D / 4), c4 = e - r * (D / 4);
+    const float4 *src = reinterpret_cast<const float4 *>(ao + (size_t)r * D) + c4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < ns; s0 += 8) {
+      float4 x[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        x[u] = s0 + u < ns ? __ldcg(src + (size_t)(s0 + u) * 8 * (D / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float wgt = s0 + u < ns ? s_w[r * kMaxSplits + s0 + u] : 0.f;
+        acc.x = fmaf(wgt, x[u].x, acc.x); acc.y = fmaf(wgt, x[u].y, acc.y);
+        acc.z = fmaf(wgt, x[u].z, acc.z); acc.w = fmaf(wgt, x[u].w, acc.w);
+      }
+    }
+    __nv_bfloat162 *dst = reinterpret_cast<__nv_bfloat162 *>(out + (qrow0 + r) * D + c4 * 4);
+    dst[0] = __floats2bfloat162_rn(acc.x, acc.y);
+    dst[1] = __floats2bfloat162_rn(acc.z, acc.w);
   }
 }
 

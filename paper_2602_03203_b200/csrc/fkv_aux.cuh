@@ -159,8 +159,8 @@ __global__ void k_append(Ctx c, int layer, const uint8_t *k, const uint8_t *v, c
 // ---------------------------------------------------------------- plan
 // One block sizes the step for segments of layers [l0, l1): which segments
 // take part, their counts, the score-tile prefix, and - when the step
-// compacts - one batch of fresh pages per segment, taken from the top of the
-// free stack and written to pt_new.  Everything later kernels need comes from
+// compacts - one batch of fresh pages per segment, reserved at the top of the
+// free stack (offset pad0 of its plan entry).  Everything later kernels need comes from
 // here, so the host never reads a length back.
 enum { PLAN_EVICT = 0, PLAN_SCORE_ALL = 1, PLAN_SELECT = 2, PLAN_COMPACT = 3 };
 
@@ -205,7 +205,9 @@ __global__ void __launch_bounds__(1024) k_plan(Ctx c, int l0, int l1, int mode, 
     }
   }
   __syncthreads();
-  const int top = c.ctrl[CTRL_FREE_TOP];
+  if (threadIdx.x == 0) s_scan[0] = c.ctrl[CTRL_FREE_TOP];
+  __syncthreads();
+  const int top = s_scan[0];
   const bool exhausted = carry_new > top;
   if (exhausted || s_fail) {
     // Not enough pages (or bad counts): make the whole step a no-op.
@@ -223,18 +225,9 @@ __global__ void __launch_bounds__(1024) k_plan(Ctx c, int l0, int l1, int mode, 
     c.planhdr[PH_NEW_PAGES] = carry_new; c.planhdr[PH_OLD_PAGES] = carry_old;
     c.planhdr[PH_PUSH_START] = top - carry_new;
   }
-  if (carry_new > 0) {
-    // Segment by segment, copy its batch of fresh page ids from the stack to pt_new.
-    for (int i = 0; i < nseg; ++i) {
-      const SegPlan p = c.plan[seg0 + i];
-      if (!p.active) continue;
-      const int cnt = (p.n_new + kPage - 1) / kPage;
-      int *dst = c.pt_new + (size_t)(seg0 + i) * c.max_pages;
-      for (int j = threadIdx.x; j < cnt; j += blockDim.x) dst[j] = c.free_stack[top - 1 - (p.pad0 + j)];
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) c.ctrl[CTRL_FREE_TOP] = top - carry_new;
-  }
+  // The fresh page ids stay on the stack above the new top until the selection kernel (or
+  // k_fill_pt_new) copies each segment's batch into pt_new; the commit pushes old pages only after that.
+  if (carry_new > 0 && threadIdx.x == 0) c.ctrl[CTRL_FREE_TOP] = top - carry_new;
 }
 
 // ---------------------------------------------------------------- commit

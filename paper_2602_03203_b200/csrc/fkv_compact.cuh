@@ -3,86 +3,73 @@
 // and position id move together from the old pages into fresh pages, so the
 // gather never overwrites a row it still has to read.
 //
-// Roofline: HBM, 2 x (4D + 4F + 4) bytes per kept pair.  grid (tiles of 32
-// output rows, work list); a warp moves 4 rows: all loads first, then all
-// stores, 16 bytes per lane for K and V.  The 16-byte chunks are re-swizzled
-// for the new row index on the way.
+// Roofline: HBM, 2 x (4D + 4F + 4) bytes per kept pair.  grid (tiles of 64
+// output rows, work list).  The CTA first resolves index and page-table
+// lookups for all its rows in one step, then every warp moves 8 rows: all
+// loads first, then all stores, 16 bytes per lane for K and V.  The 16-byte
+// chunks are re-swizzled for the new row index on the way.
 #pragma once
 #include "fkv_dev.cuh"
 
 namespace fkv {
 
-constexpr int kCompactRows = 32;  // output rows per CTA (two pages)
+constexpr int kCompactRows = 64;  // output rows per CTA (four pages)
+constexpr int kCompactRPW = 8;    // rows per warp, all loaded before any is stored
 
 template <int D>
 __global__ void __launch_bounds__(256) k_compact(Ctx c, const int32_t *idx, int seg_base) {
   constexpr int NCH = D / 8;               // 16-byte chunks per K (or V) row
-  constexpr int QPL = (2 * NCH + 31) / 32;  // chunks per lane (1 for D = 128 and 64)
+  static_assert(2 * NCH <= 32, "one chunk per lane");
+  __shared__ long long s_src[kCompactRows];  // physical source slot (page * 16 + row) or -1
+  __shared__ int s_dst[kCompactRows / kPage];
   if ((int)blockIdx.y >= c.planhdr[PH_NWORK]) return;
   const int seg = c.work[blockIdx.y];
   const SegPlan p = c.plan[seg];
   if (!p.active) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int j0 = blockIdx.x * kCompactRows + warp * 4;
+  const int j0 = blockIdx.x * kCompactRows;
   if (j0 >= p.n_new) return;
-  const int32_t *ix = idx + (size_t)(seg - seg_base) * c.cap;
-  const int *ptold = c.pt + (size_t)seg * c.max_pages, *ptnew = c.pt_new + (size_t)seg * c.max_pages;
-  const int FH = c.F >> 1;  // 8-byte feature chunks per row
-
-  const uint8_t *src[4];
-  int sr[4];
-  bool ok[4];
-#pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    const int j = j0 + u;
-    ok[u] = j < p.n_new;
-    int s = ok[u] ? ix[j] : 0;
-    if (ok[u] && (s < 0 || s >= p.n_old)) {
-      if (lane == 0) set_status(c, kDevBadIndex);
-      ok[u] = false;
-      s = 0;
+  // Phase 1: one index and one page-table lookup per output row, all rows of the CTA at once.
+  if (threadIdx.x < kCompactRows) {
+    const int j = j0 + threadIdx.x;
+    long long src = -1;
+    if (j < p.n_new) {
+      const int s = idx[(size_t)(seg - seg_base) * c.cap + j];
+      if (s < 0 || s >= p.n_old) set_status(c, kDevBadIndex);
+      else src = (long long)c.pt[(size_t)seg * c.max_pages + s / kPage] * kPage + s % kPage;
     }
-    sr[u] = s % kPage;
-    src[u] = c.pool + (size_t)ptold[s / kPage] * c.page_bytes;
+    s_src[threadIdx.x] = src;
+  } else if (threadIdx.x < kCompactRows + kCompactRows / kPage) {
+    const int q = threadIdx.x - kCompactRows, pg = j0 / kPage + q;
+    s_dst[q] = pg * kPage < p.n_new ? c.pt_new[(size_t)seg * c.max_pages + pg] : -1;
   }
-  uint4 kv[4][QPL];
-  float2 ft[4][2];
-  int32_t ps[4];
+  __syncthreads();
+  // Phase 2: each warp moves 8 rows; lane = one 16-byte chunk of K (0..NCH-1) or V.
+  const int FH = c.F >> 1;  // 8-byte feature chunks per row (<= 24)
+  const int isv = lane >= NCH, ch = isv ? lane - NCH : lane;
+  const bool kvlane = lane < 2 * NCH;
+  uint4 kv[kCompactRPW];
+  float2 ft[kCompactRPW];
+  int32_t ps[kCompactRPW];
+  const int r0 = warp * kCompactRPW;
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    if (!ok[u]) continue;
-#pragma unroll
-    for (int q = 0; q < QPL; ++q) {
-      const int ch2 = lane + q * 32;
-      if (ch2 < 2 * NCH) {
-        const int isv = ch2 >= NCH, ch = isv ? ch2 - NCH : ch2;
-        kv[u][q] = *reinterpret_cast<const uint4 *>(src[u] + (isv ? c.off_v : 0) + kv_chunk_off(sr[u], ch));
-      }
-    }
-    const float2 *f = reinterpret_cast<const float2 *>(src[u] + c.off_f) + sr[u] * FH;
-#pragma unroll
-    for (int q = 0; q < 2; ++q)
-      if (lane + q * 32 < FH) ft[u][q] = f[lane + q * 32];
-    if (lane == 31) ps[u] = reinterpret_cast<const int32_t *>(src[u] + c.off_p)[sr[u]];
+  for (int u = 0; u < kCompactRPW; ++u) {
+    const long long src = s_src[r0 + u];
+    if (src < 0) continue;
+    const uint8_t *page = c.pool + (size_t)(src / kPage) * c.page_bytes;
+    const int sr = (int)(src % kPage);
+    if (kvlane) kv[u] = *reinterpret_cast<const uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(sr, ch));
+    if (lane < FH) ft[u] = reinterpret_cast<const float2 *>(page + c.off_f)[sr * FH + lane];
+    if (lane == 31) ps[u] = reinterpret_cast<const int32_t *>(page + c.off_p)[sr];
   }
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    if (!ok[u]) continue;
-    const int j = j0 + u, dr = j % kPage;
-    uint8_t *dst = c.pool + (size_t)ptnew[j / kPage] * c.page_bytes;
-#pragma unroll
-    for (int q = 0; q < QPL; ++q) {
-      const int ch2 = lane + q * 32;
-      if (ch2 < 2 * NCH) {
-        const int isv = ch2 >= NCH, ch = isv ? ch2 - NCH : ch2;
-        *reinterpret_cast<uint4 *>(dst + (isv ? c.off_v : 0) + kv_chunk_off(dr, ch)) = kv[u][q];
-      }
-    }
-    float2 *f = reinterpret_cast<float2 *>(dst + c.off_f) + dr * FH;
-#pragma unroll
-    for (int q = 0; q < 2; ++q)
-      if (lane + q * 32 < FH) f[lane + q * 32] = ft[u][q];
-    if (lane == 31) reinterpret_cast<int32_t *>(dst + c.off_p)[dr] = ps[u];
+  for (int u = 0; u < kCompactRPW; ++u) {
+    if (s_src[r0 + u] < 0) continue;
+    const int jr = r0 + u, dr = jr % kPage;
+    uint8_t *page = c.pool + (size_t)s_dst[jr / kPage] * c.page_bytes;
+    if (kvlane) *reinterpret_cast<uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(dr, ch)) = kv[u];
+    if (lane < FH) reinterpret_cast<float2 *>(page + c.off_f)[dr * FH + lane] = ft[u];
+    if (lane == 31) reinterpret_cast<int32_t *>(page + c.off_p)[dr] = ps[u];
   }
 }
 

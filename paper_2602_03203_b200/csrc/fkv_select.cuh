@@ -4,10 +4,10 @@
 // are written in ascending order, which is the order compaction needs.
 //
 // Integer work on 4 bytes per pair, read from L2 right after the scorer wrote
-// them.  One CTA per segment: a 4 x 8-bit most-significant-digit radix select
-// finds the k-th largest key T and how many pairs equal to T are still needed;
-// one ordered pass then emits {key > T} plus the first `need` slots with
-// key == T, using block prefix sums - no atomics decide which tied pair stays.
+// them.  One CTA per segment: a histogram select finds the k-th largest key T
+// and how many pairs equal to T are still needed; one ordered pass then emits
+// {key > T} plus the first `need` slots with key == T, using block prefix
+// sums - no atomics decide which tied pair stays.
 #pragma once
 #include "fkv_dev.cuh"
 
@@ -23,18 +23,51 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 }
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelBins = 2048;
+
+// Fresh page ids of one compacted segment: copied from the batch the planner
+// reserved at the top of the free stack into the segment's row of pt_new.
+__device__ __forceinline__ void fill_pt_new(const Ctx &c, int seg, const SegPlan &p) {
+  if (!p.active) return;
+  const int top0 = c.planhdr[PH_PUSH_START] + c.planhdr[PH_NEW_PAGES];  // stack top before the planner took them
+  const int cnt = (p.n_new + kPage - 1) / kPage;
+  int *dst = c.pt_new + (size_t)seg * c.max_pages;
+  for (int j = threadIdx.x; j < cnt; j += blockDim.x) dst[j] = c.free_stack[top0 - 1 - (p.pad0 + j)];
+}
+
+// grid = segments of the call: pt_new rows when no selection kernel runs (fkv_compact).
+__global__ void k_fill_pt_new(Ctx c, int seg0, int nseg) {
+  if ((int)blockIdx.x < nseg) fill_pt_new(c, seg0 + blockIdx.x, c.plan[seg0 + blockIdx.x]);
+}
 
 // scores/idx: row (seg - seg_base) * cap.  kept_count (optional): [seg - seg_base].
+//
+// Every thread owns 32 consecutive slots per round of 32768 (so one block
+// prefix sum orders a whole round).  SINGLE = the segment fits one round: the
+// keys are loaded once and stay in registers for every pass.  Otherwise each
+// pass streams the rounds again from L2, 8 loads in flight per thread.
+//
+// Selection of the k-th largest key T: a min/max pass fixes the key window;
+// each histogram pass splits the current window into up to 2048 equal bins
+// (so the bins follow the data, not fixed bit fields, and shared-memory
+// atomics spread out), picks the bin where the count from the top crosses k,
+// and narrows the window to it - at most three passes for 32-bit keys.
+constexpr int kSelPerThread = 32;
+constexpr int kSelRound = kSelThreads * kSelPerThread;
+
+template <bool SINGLE>
 __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scores, int32_t *idx, int32_t *kept_count,
-                                                         int seg_base) {
-  __shared__ unsigned s_hist[256];
+                                                         int seg_base, int fill_pages) {
+  __shared__ unsigned s_hist[kSelBins];
   __shared__ int s_scan[33];
-  __shared__ unsigned s_digit, s_krem;
+  __shared__ unsigned s_red[64];
+  __shared__ unsigned s_bin, s_krem;
   __shared__ unsigned long long s_wsum[33];
   if ((int)blockIdx.x >= c.planhdr[PH_NWORK]) return;
   const int seg = c.work[blockIdx.x];
   const SegPlan p = c.plan[seg];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (fill_pages) fill_pt_new(c, seg, p);
   const int m = p.n_old - p.r, k = p.k_sel;
   const float *sc = scores + (size_t)(seg - seg_base) * c.cap;
   int32_t *out = idx + (size_t)(seg - seg_base) * c.cap;
@@ -46,62 +79,90 @@ __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scor
     for (int j = tid; j < m; j += kSelThreads) out[j] = j;
     return;
   }
-
-  // ---- radix select of the k-th largest key ----
-  uint32_t prefix = 0, mask = 0;
-  unsigned krem = (unsigned)k;
-  const float4 *sc4 = reinterpret_cast<const float4 *>(sc);
-  const int m4 = (m + 3) >> 2;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    if (tid < 256) s_hist[tid] = 0;
-    __syncthreads();
-    for (int i = tid; i < ((m4 + kSelThreads - 1) / kSelThreads) * kSelThreads; i += kSelThreads) {
-      float4 x = i < m4 ? sc4[i] : make_float4(0, 0, 0, 0);
-      const float xs[4] = {x.x, x.y, x.z, x.w};
+  const int rounds = SINGLE ? 1 : (m + kSelRound - 1) / kSelRound;
+  uint32_t key[kSelPerThread];
+  int nv = 0;  // valid keys of this thread in the loaded round (they are its first nv)
+  auto load_round = [&](int round) {
+    const int base = round * kSelRound + tid * kSelPerThread;
+    nv = min(max(m - base, 0), kSelPerThread);
+    const float4 *src = reinterpret_cast<const float4 *>(sc + base);
+    float4 x[kSelPerThread / 4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const uint32_t key = score_key(xs[e]);
-        const bool valid = (i * 4 + e) < m && (key & mask) == prefix;
-        // One shared-memory atomic per distinct digit in the warp.
-        const unsigned digit = valid ? ((key >> shift) & 255u) : 0xffffffffu;
-        const unsigned peers = __match_any_sync(0xffffffffu, digit);
-        if (valid && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[digit], (unsigned)__popc(peers));
-      }
+    for (int q = 0; q < kSelPerThread / 4; ++q) x[q] = q * 4 < nv ? src[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int q = 0; q < kSelPerThread / 4; ++q) {
+      key[4 * q] = score_key(x[q].x); key[4 * q + 1] = score_key(x[q].y);
+      key[4 * q + 2] = score_key(x[q].z); key[4 * q + 3] = score_key(x[q].w);
     }
-    __syncthreads();
-    // Digit d is chosen when (#keys with a larger digit) < krem <= (that + hist[d]).
-    {
-      const int v = tid < 256 ? (int)s_hist[255 - tid] : 0;  // descending digits
-      int tot;
-      const int above = block_excl_scan(v, s_scan, tot);
-      if (tid < 256 && (unsigned)above < krem && krem <= (unsigned)(above + v)) {
-        s_digit = 255u - tid;
-        s_krem = krem - (unsigned)above;
-      }
-    }
-    __syncthreads();
-    prefix |= s_digit << shift;
-    mask |= 255u << shift;
-    krem = s_krem;
-    __syncthreads();
+  };
+  if (SINGLE) load_round(0);
+
+  // ---- key window ----
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
+  for (int round = 0; round < rounds; ++round) {
+    if (!SINGLE) load_round(round);
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j)
+      if (j < nv) { kmin = min(kmin, key[j]); kmax = max(kmax, key[j]); }
   }
-  const uint32_t T = prefix;
-  const unsigned need = krem;  // pairs with key == T still to keep, lowest slots first
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) { s_red[warp] = kmin; s_red[32 + warp] = kmax; }
+  __syncthreads();
+  kmin = __reduce_min_sync(0xffffffffu, s_red[lane]);
+  kmax = __reduce_max_sync(0xffffffffu, s_red[32 + lane]);
 
-  // ---- ordered emit ----
-  unsigned run_gt = 0, run_eq = 0;
-  for (int base = 0; base < m4; base += kSelThreads) {
-    const int i = base + tid;
-    float4 x = i < m4 ? sc4[i] : make_float4(0, 0, 0, 0);
-    const float xs[4] = {x.x, x.y, x.z, x.w};
-    unsigned gt[4], eq[4], cgt = 0, ceq = 0;
+  uint32_t T = kmin;
+  unsigned need = (unsigned)k;
+  if (kmin != kmax) {
+    uint32_t lo = kmin, wmax = kmax - kmin;  // window: keys with key - lo <= wmax
+    unsigned krem = (unsigned)k;
+    int bits = 32 - __clz(wmax);
+    for (;;) {
+      const int shift = bits > 11 ? bits - 11 : 0;
+      for (int b = tid; b < kSelBins; b += kSelThreads) s_hist[b] = 0;
+      __syncthreads();
+      for (int round = 0; round < rounds; ++round) {
+        if (!SINGLE) load_round(round);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const uint32_t key = score_key(xs[e]);
-      const bool in = (i * 4 + e) < m;
-      gt[e] = in && key > T; eq[e] = in && key == T;
-      cgt += gt[e]; ceq += eq[e];
+        for (int j = 0; j < kSelPerThread; ++j) {
+          const uint32_t d = key[j] - lo;
+          if (j < nv && key[j] >= lo && d <= wmax) atomicAdd(&s_hist[d >> shift], 1u);
+        }
+      }
+      __syncthreads();
+      // Bins in descending order, two per thread: 2047 - 2 tid, then 2046 - 2 tid.
+      {
+        const unsigned v0 = s_hist[kSelBins - 1 - 2 * tid], v1 = s_hist[kSelBins - 2 - 2 * tid];
+        int tot;
+        const unsigned above = (unsigned)block_excl_scan((int)(v0 + v1), s_scan, tot);
+        if (above < krem && krem <= above + v0) {
+          s_bin = kSelBins - 1 - 2 * tid; s_krem = krem - above;
+        } else if (above + v0 < krem && krem <= above + v0 + v1) {
+          s_bin = kSelBins - 2 - 2 * tid; s_krem = krem - above - v0;
+        }
+      }
+      __syncthreads();
+      lo += s_bin << shift;
+      krem = s_krem;
+      __syncthreads();
+      if (shift == 0) break;
+      wmax = (1u << shift) - 1u;
+      bits = shift;
+    }
+    T = lo;
+    need = krem;  // pairs with key == T still to keep, lowest slots first
+  }
+
+  // ---- ordered emit: one block prefix sum per round ----
+  unsigned run_gt = 0, run_eq = 0;
+  for (int round = 0; round < rounds; ++round) {
+    if (!SINGLE) load_round(round);
+    unsigned cgt = 0, ceq = 0;
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j) {
+      cgt += (j < nv && key[j] > T);
+      ceq += (j < nv && key[j] == T);
     }
     // Exclusive block scan of (cgt, ceq) packed in 64 bits.
     unsigned long long v = (unsigned long long)cgt | ((unsigned long long)ceq << 32), inc = v;
@@ -126,11 +187,13 @@ __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scor
     __syncthreads();
     const unsigned long long excl = s_wsum[warp] + inc - v, tot = s_wsum[32];
     unsigned bgt = run_gt + (unsigned)(excl & 0xffffffffu), beq = run_eq + (unsigned)(excl >> 32);
+    const int slot0 = round * kSelRound + tid * kSelPerThread;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      if (gt[e]) out[bgt + min(beq, need)] = i * 4 + e;
-      else if (eq[e] && beq < need) out[bgt + beq] = i * 4 + e;
-      bgt += gt[e]; beq += eq[e];
+    for (int j = 0; j < kSelPerThread; ++j) {
+      const bool g = j < nv && key[j] > T, e = j < nv && key[j] == T;
+      if (g) out[bgt + min(beq, need)] = slot0 + j;
+      else if (e && beq < need) out[bgt + beq] = slot0 + j;
+      bgt += g; beq += e;
     }
     run_gt += (unsigned)(tot & 0xffffffffu);
     run_eq += (unsigned)(tot >> 32);
