@@ -248,6 +248,25 @@ def decode_attn_dense_noalloc(q, k, v, group_size, out=None, scale=0.0):
     return out
 
 
+def pages_for(w, num_layers=None, extra_tokens=256) -> int:
+    """Pool pages that hold every sequence of `w` at its own length plus `extra_tokens`, and the
+    fresh pages an all-layer eviction takes before it returns the old ones."""
+    L = num_layers or w.num_layers
+    per_head = sum(-(-(n + extra_tokens) // w.page_size) + -(-min(b, n) // w.page_size) + 1
+                   for n, b in zip(w.lens, w.budgets))
+    return L * w.num_kv_heads * per_head
+
+
+def workspace_bytes_for(w, num_layers=None, num_pages=0, max_tokens=None) -> int:
+    """Bytes of device workspace ``from_workload`` would allocate (no device access)."""
+    cfg = FkvConfig(num_layers or w.num_layers, w.num_kv_heads, w.group_size, w.head_dim, w.batch, w.page_size,
+                    w.scorer_hidden, w.activation, max(w.budgets), w.recent_keep,
+                    max_tokens or (max(w.lens) + 256), num_pages)
+    nbytes = ctypes.c_size_t(0)
+    _check(lib().fkv_workspace_bytes(ctypes.byref(cfg), ctypes.byref(nbytes)), "fkv_workspace_bytes")
+    return nbytes.value
+
+
 def from_workload(w, num_layers=None, num_pages=0, max_tokens=None) -> Cache:
     """A cache shaped for a ``workloads.Workload`` with per-sequence budgets set."""
     L = num_layers or w.num_layers

@@ -1,0 +1,248 @@
+"""Full-size parity: the five configurations at (or sliced from) their real sizes, in the launch
+configuration the benchmark times (one all-layer eviction, decode attention per layer), checked
+against the CPU oracle on SAMPLED segments the oracle computes one by one, plus properties that
+hold at any size (kept count, strictly increasing positions, recent window, page accounting).
+
+Inputs are generated on the GPU (the CPU generator would take minutes at these sizes); the
+sampled segments are copied to the host, so both sides still see the same bytes.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from harness import kept_set_within_band
+from paper_2602_03203_b200 import binding, workloads as wl
+from util import bits, bits_to_f64, npf
+
+pytestmark = pytest.mark.gpu
+
+SCORE_TOL = 1e-3
+ATTN_TOL = 2e-2
+
+
+class BigLoaded:
+    """A workload resident in a cache; host copies kept only for the sampled (layer, seq) pairs."""
+
+    def __init__(self, w, num_layers, samples, extra_tokens=256):
+        self.w, self.L = w, num_layers
+        free, _ = torch.cuda.mem_get_info()
+        self.cache = None
+        pages = binding.pages_for(w, num_layers, extra_tokens)
+        need = binding.workspace_bytes_for(w, num_layers, num_pages=pages, max_tokens=max(w.lens) + extra_tokens)
+        if need * 1.3 > free:     # workspace + generator scratch
+            pytest.skip(f"needs {need * 1.3 / 1e9:.1f} GB of device memory, {free / 1e9:.1f} GB free")
+        self.cache = binding.from_workload(w, num_layers, num_pages=pages, max_tokens=max(w.lens) + extra_tokens)
+        self.seg, self.scorer = {}, {}
+        want = {(l, s) for l, s, _ in samples}
+        for l in range(num_layers):
+            W1, b1, W2, b2 = wl.scorer_params(w, l, "cuda")
+            self.cache.load_scorers(l, W1, b1, W2, b2)
+            if any(l == ll for ll, _ in want):
+                self.scorer[l] = tuple(npf(t) for t in (W1, b1, W2, b2))
+            for s in range(w.batch):
+                K, V, A, pos = wl.layer_inputs(w, l, s, "cuda")
+                self.cache.prefill(l, s, K, V, A, pos)
+                if (l, s) in want:
+                    self.seg[(l, s)] = dict(K=bits(K), V=bits(V), A=npf(A), pos=npf(pos))
+                del K, V, A, pos
+        torch.cuda.synchronize()
+
+    def head(self, l, s, h):
+        d = self.seg[(l, s)]
+        return d["K"][h], d["V"][h], d["A"][h], d["pos"]
+
+    def weights(self, l, h):
+        W1, b1, W2, b2 = self.scorer[l]
+        return W1[h], b1[h], W2[h], float(b2[h])
+
+    def export(self, l, s, h):
+        k, v, a, p = self.cache.export_head(l, s, h)
+        return bits(k), bits(v), npf(a), npf(p)
+
+
+def check_evicted_segment(ld, l, s, h, gpu_scores):
+    """One sampled segment after the eviction: scores, kept set, moved rows."""
+    w = ld.w
+    n, B, R = w.lens[s], w.budgets[s], w.recent_keep
+    K, V, A, pos = ld.head(l, s, h)
+    phi = oracle.score(K, V, A, *ld.weights(l, h), act=w.activation)
+    assert np.abs(phi - gpu_scores[:n]).max() <= SCORE_TOL
+    k2, v2, a2, p2 = ld.export(l, s, h)
+    assert len(p2) == min(B, n) and np.all(np.diff(p2) > 0)
+    kept_g = np.searchsorted(pos, p2).astype(np.int32)
+    assert np.array_equal(pos[kept_g], p2)
+    assert np.array_equal(kept_g, oracle.select(gpu_scores[:n], B, R))          # bit-exact from identical scores
+    assert kept_set_within_band(phi, oracle.select(phi, B, R), kept_g, n, B, R, SCORE_TOL)
+    Ko, Vo, Ao, po = oracle.compact(K, V, A, pos, kept_g)
+    assert np.array_equal(k2, Ko) and np.array_equal(v2, Vo) and np.array_equal(a2, Ao) and np.array_equal(p2, po)
+    return k2, v2
+
+
+def check_attention(ld, l, samples, step=0):
+    w, g = ld.w, ld.w.group_size
+    q = wl.queries(w, l, step, "cuda")
+    out = ld.cache.decode_attn(l, q)
+    torch.cuda.synchronize()
+    ob, qb = bits(out), bits(q)
+    for s, h in samples:
+        k2, v2, _, _ = ld.export(l, s, h)
+        ref, ref64 = oracle.attend(qb[s, h * g:(h + 1) * g], k2, v2)
+        err = np.abs(bits_to_f64(ob[s, h * g:(h + 1) * g]) - bits_to_f64(ref))
+        assert np.all(err <= np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64)))
+    assert torch.isfinite(out.float()).all()
+
+
+def all_layers_properties(ld):
+    """Size-independent checks over EVERY segment, on the device: counts and position order."""
+    w = ld.w
+    for l in range(ld.L):
+        assert ld.cache.lengths(l) == [min(b, n) for b, n in zip(w.budgets, w.lens)]
+    for l in range(0, ld.L, max(1, ld.L // 6)):
+        for s in range(0, w.batch, max(1, w.batch // 4)):
+            for h in range(w.num_kv_heads):
+                _, _, _, p = ld.cache.export_head(l, s, h)
+                assert bool((p[1:] > p[:-1]).all()) and int(p[-1]) < w.lens[s]
+                if w.recent_keep:
+                    r = min(w.recent_keep, len(p))
+                    assert p[-r:].tolist() == list(range(w.lens[s] - r, w.lens[s]))
+
+
+@pytest.mark.parametrize("budget", [2048, 8192, 16384])
+def test_config3_full_size(budget):
+    # 36 layers x 8 KV heads x 32768 pairs, one all-layer eviction: exactly what the benchmark times.
+    w = wl.config(3, budget=budget)
+    samples = [(0, 0, 0), (17, 0, 3), (35, 0, 7)]
+    ld = BigLoaded(w, w.num_layers, samples)
+    free0 = ld.cache.device_status()[1]
+    gs = {l: ld.cache.score(l)[s, h].cpu().numpy() for l, s, h in samples}
+    ld.cache.evict(binding.ALL_LAYERS)
+    for l, s, h in samples:
+        check_evicted_segment(ld, l, s, h, gs[l])
+    all_layers_properties(ld)
+    status, free1 = ld.cache.device_status()
+    assert status == 0
+    segs = w.num_layers * w.num_kv_heads
+    assert free1 - free0 == segs * (32768 // 16 - budget // 16)
+    for l, s, h in samples:
+        check_attention(ld, l, [(s, h)])
+    # decode continues on the compacted cache: 3 tokens through all layers, then attention again
+    for step in range(3):
+        for l in range(ld.L):
+            k, v = wl.new_kv(w, l, step, "cuda")
+            ld.cache.append(l, k, v)
+    assert ld.cache.lengths(35) == [budget + 3]
+    check_attention(ld, 35, [(0, 7)], step=1)
+    assert ld.cache.device_status()[0] == 0
+
+
+def test_config2_full_schedule():
+    # 36 layers, 8320 -> 4096 with the recent 128 protected, then the 1024-step schedule:
+    # append + attention in every layer, an all-layer eviction every 128 tokens (8 events).
+    w = wl.config(2)
+    B, Lev = w.budgets[0], w.recent_keep
+    samples = [(0, 0, 1), (20, 0, 6)]
+    ld = BigLoaded(w, w.num_layers, samples, extra_tokens=512)
+    gs = {l: ld.cache.score(l)[s, h].cpu().numpy() for l, s, h in samples}
+    ld.cache.evict(binding.ALL_LAYERS)
+    state = {}
+    for l, s, h in samples:
+        K, V, A, pos = ld.head(l, s, h)
+        check_evicted_segment(ld, l, s, h, gs[l])
+        k2, v2, a2, p2 = ld.export(l, s, h)
+        assert p2[-Lev:].tolist() == list(range(w.lens[0] - Lev, w.lens[0]))
+        state[(l, h)] = [k2, v2, a2, p2]
+    all_layers_properties(ld)
+    steps = 1024
+    Lw = w.num_layers
+    for step in range(steps):
+        kk = torch.stack([torch.stack(wl.new_kv(w, l, step, "cuda")) for l in range(Lw)])   # [L][2][1][Hkv][D]
+        k_all, v_all = kk[:, 0].contiguous(), kk[:, 1].contiguous()
+        q_all = torch.stack([wl.queries(w, l, step, "cuda") for l in range(Lw)])
+        out = ld.cache.decode_step(k_all, v_all, q_all)
+        kb, vb = bits(k_all), bits(v_all)
+        for (l, h), st in state.items():
+            st[0] = np.concatenate([st[0], kb[l, 0, h][None]]); st[1] = np.concatenate([st[1], vb[l, 0, h][None]])
+            st[2] = np.concatenate([st[2], np.zeros((1, st[2].shape[1]), np.float32)])
+            st[3] = np.concatenate([st[3], [st[3][-1] + 1]]).astype(np.int32)
+        if step in (0, 500, steps - 1):      # attention over the growing cache, sampled heads
+            ob, qb = bits(out), bits(q_all)
+            g = w.group_size
+            for (l, h), st in state.items():
+                ref, ref64 = oracle.attend(qb[l, 0, h * g:(h + 1) * g], st[0], st[1])
+                err = np.abs(bits_to_f64(ob[l, 0, h * g:(h + 1) * g]) - bits_to_f64(ref))
+                assert np.all(err <= np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64)))
+        if (step + 1) % Lev == 0:
+            assert ld.cache.lengths(0) == [B + Lev]
+            ld.cache.evict(binding.ALL_LAYERS)
+            assert ld.cache.lengths(0) == [B] and ld.cache.lengths(Lw - 1) == [B]
+            for (l, h), (K, V, A, pos) in list(state.items()):
+                phi = oracle.score(K, V, A, *ld.weights(l, h))
+                k2, v2, a2, p2 = ld.export(l, 0, h)
+                kept_g = np.searchsorted(pos, p2).astype(np.int32)
+                assert np.array_equal(pos[kept_g], p2)
+                assert kept_set_within_band(phi, oracle.select(phi, B, Lev), kept_g, len(pos), B, Lev, SCORE_TOL)
+                assert kept_g[-Lev:].tolist() == list(range(len(pos) - Lev, len(pos)))
+                assert np.array_equal(k2, K[kept_g]) and np.array_equal(a2, A[kept_g])
+                state[(l, h)] = [K[kept_g], V[kept_g], A[kept_g], pos[kept_g]]
+    assert ld.cache.device_status()[0] == 0
+
+
+def test_config4_full_size():
+    # 28 layers x 16 sequences of different lengths x 4 KV heads, group of 7, B = len / 2.
+    w = wl.config(4)
+    longest, shortest = int(np.argmax(w.lens)), int(np.argmin(w.lens))
+    samples = [(0, longest, 0), (13, shortest, 2), (27, 5, 3)]
+    ld = BigLoaded(w, w.num_layers, samples)
+    gs = {(l, s, h): ld.cache.score(l)[s, h].cpu().numpy() for l, s, h in samples}
+    ld.cache.evict(binding.ALL_LAYERS)
+    for l, s, h in samples:
+        check_evicted_segment(ld, l, s, h, gs[(l, s, h)])
+    all_layers_properties(ld)
+    for l, s, h in samples:
+        check_attention(ld, l, [(s, h)])
+    assert ld.cache.device_status()[0] == 0
+
+
+def test_config5_layer_slice():
+    # 8 sequences x 8 KV heads x 65536 pairs, B = 16384, exact duplicate rows (1 %): a slice of
+    # 4 of the 32 layers (the per-layer shapes, and so every launch, are those of the full config).
+    w = wl.config(5)
+    samples = [(0, 0, 0), (3, 7, 5)]
+    ld = BigLoaded(w, 4, samples)
+    gs = {(l, s, h): ld.cache.score(l)[s, h].cpu().numpy() for l, s, h in samples}
+    for (l, s, h), sc in gs.items():           # duplicates tie bit for bit
+        K, V, A, _ = ld.head(l, s, h)
+        rows = np.concatenate([K.astype(np.uint32), V.astype(np.uint32), A.view(np.uint32)], axis=1)
+        _, inv, cnt = np.unique(rows, axis=0, return_inverse=True, return_counts=True)
+        inv = inv.reshape(-1)
+        u = sc[:w.lens[s]].view(np.uint32)
+        for gidx in np.where(cnt > 1)[0][:200]:
+            assert len(set(u[inv == gidx].tolist())) == 1
+    ld.cache.evict(binding.ALL_LAYERS)
+    for l, s, h in samples:
+        check_evicted_segment(ld, l, s, h, gs[(l, s, h)])
+    all_layers_properties(ld)
+    for l, s, h in samples:
+        check_attention(ld, l, [(s, h)])
+    assert ld.cache.device_status()[0] == 0
+
+
+@pytest.mark.parametrize("n,B,R", [(40000, 10000, 0), (65536, 16384, 0), (70001, 3, 5), (32769, 32768, 0),
+                                   (65536, 16384, 256)])
+def test_select_long_segments_bit_exact(n, B, R):
+    # Segments longer than one selection round (32768 keys): the multi-round path.
+    w = wl.Workload("sel_long", 1, 2, 4, 64, (n,), (B,), R, 12, "normal")
+    c = binding.from_workload(w)
+    K, V, A, pos = wl.layer_inputs(w, 0, 0, "cuda")
+    c.prefill(0, 0, K, V, A, pos)
+    rng = np.random.default_rng(n + B)
+    sc = np.full((1, 2, c.cap), np.nan, np.float32)
+    sc[0, 0, :n] = rng.standard_normal(n).astype(np.float32)
+    sc[0, 1, :n] = (np.round(rng.standard_normal(n) * 8) / 8).astype(np.float32)      # heavy ties
+    idx, cnt = c.select(0, torch.from_numpy(sc).cuda())
+    idx, cnt = npf(idx), npf(cnt)
+    for h in range(2):
+        ref = oracle.select(sc[0, h, :n], B, R)
+        assert cnt[0, h] == len(ref) and np.array_equal(idx[0, h, :len(ref)], ref)
+    assert c.device_status()[0] == 0
