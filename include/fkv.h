@@ -149,12 +149,25 @@ int fkv_evict(fkv_cache *c, int layer, void *stream);
 int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream);
 
 /*
+ * append(k, v) followed by decode_attn(q) on `layer`, as ONE kernel launch
+ * (Section 3.1 + Appendix A): the new pair of every participating sequence is
+ * stored at slot n and attended together with the n retained pairs.  Arguments
+ * as in fkv_append and fkv_decode_attn; the result equals the two calls made
+ * one after the other.
+ */
+int fkv_append_decode_attn(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos,
+                           uint64_t seq_mask, const void *q, void *out, float scale, void *stream);
+
+/*
  * One decode token through every layer, in layer order: for l = 0 .. L-1,
- * append(k[l], v[l]) then decode_attn(q[l]) -> out[l].  k, v: dev
+ * fkv_append_decode_attn(k[l], v[l], q[l]) -> out[l].  k, v: dev
  * [L][max_batch][Hkv][D] bf16; q, out: dev [L][max_batch][Hkv*g][D] bf16; pos:
- * dev [max_batch] or NULL (as fkv_append).  Exactly the two calls above issued
- * L times from native code (a driver loop for engines that have all layers'
- * tensors at hand, and for benchmarks of the attention side alone).
+ * dev [max_batch] or NULL (as fkv_append).  One launch per layer, issued from
+ * native code; layer l's launch is allowed to start reading its own cache
+ * while layer l-1's launch is finishing (programmatic dependent launch; q, k,
+ * v and out of layer l are touched only after layer l-1's launch is complete).
+ * For engines that have all layers' tensors at hand, and for benchmarks of the
+ * attention side alone.
  */
 int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *pos, const void *q, void *out,
                     float scale, void *stream);

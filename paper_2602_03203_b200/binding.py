@@ -26,7 +26,7 @@ EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", 
            "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
            "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
            "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing",
-           "fkv_decode_step", "fkv_decode_attn_dense_noalloc"]
+           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn"]
 
 
 class FkvConfig(ctypes.Structure):
@@ -149,6 +149,16 @@ class Cache:
             out = torch.empty_like(q)
         _check(lib().fkv_decode_attn(self._h, layer, _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16),
                                      ctypes.c_float(scale), _stream()), "fkv_decode_attn")
+        return out
+
+    def append_decode_attn(self, layer, k, v, q, out=None, pos=None, seq_mask=0, scale=0.0):
+        """append(k, v) then decode_attn(q) on one layer, as one launch."""
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib().fkv_append_decode_attn(self._h, layer, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
+                                            _ptr(pos, torch.int32), ctypes.c_uint64(seq_mask), _ptr(q, torch.bfloat16),
+                                            _ptr(out, torch.bfloat16), ctypes.c_float(scale), _stream()),
+               "fkv_append_decode_attn")
         return out
 
     def decode_step(self, k, v, q, out=None, pos=None, scale=0.0):

@@ -36,7 +36,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, part_o, part_ml,
-      tickets, total;
+      tickets, seq_tickets, total;
   int cap, max_pages, num_pages, page_bytes, F, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
 };
 
@@ -89,6 +89,7 @@ Layout make_layout(const fkv_config &c) {
   L.part_o = take(lsegs * kMaxSplits * 8 * D * 4);
   L.part_ml = take(lsegs * kMaxSplits * 8 * 2 * 4);
   L.tickets = take(lsegs * 4);
+  L.seq_tickets = take((size_t)c.max_batch * 4);
   L.total = off;
   return L;
 }
@@ -172,18 +173,60 @@ int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, 
   return FKV_OK;
 }
 
+// One launch of the attention kernel for `layer`: optional fused append, optional overlap of its prologue with
+// the previous launch (pdl; only when that launch is known to be this kernel on ANOTHER layer).
 template <int D>
-int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale_log2, int splits, cudaStream_t st) {
+int launch_attend_t(fkv_cache *c, const AttendArgs &a, int splits, bool pdl, cudaStream_t st) {
   const size_t smem = AttendSmem::bytes(D, kAttendPPS, kAttendStages);
   static bool attr_done = false;
   if (!attr_done) {
     FKV_CUDA(cudaFuncSetAttribute(k_attend<D, kAttendPPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_done = true;
   }
-  dim3 grid(splits, c->cfg.max_batch * c->cfg.num_kv_heads);
-  k_attend<D, kAttendPPS><<<grid, (kAttendPPS + 1) * 32, smem, st>>>(
-      c->ctx, layer, (const __nv_bfloat16 *)q, (__nv_bfloat16 *)out, scale_log2, kAttendMinPages, kAttendStages);
-  FKV_LAUNCHED(c);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(splits, c->cfg.max_batch * c->cfg.num_kv_heads);
+  cfg.blockDim = dim3((kAttendPPS + 1) * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  FKV_CUDA(cudaLaunchKernelEx(&cfg, k_attend<D, kAttendPPS>, c->ctx, a));
+  ++c->launches;
+  return FKV_OK;
+}
+
+// Attention over `layer`, with the new pair of every participating sequence appended first when k_new is given.
+int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale, const void *k_new, const void *v_new,
+                  const int32_t *pos, uint64_t seq_mask, bool pdl, cudaStream_t st) {
+  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads, D = c->cfg.head_dim;
+  const bool app = k_new != nullptr;
+  long long pages = 0;
+  int maxpages = 0;
+  for (int s = 0; s < batch; ++s) {
+    const int n = c->h_len[(size_t)layer * batch + s] + ((app && (!seq_mask || ((seq_mask >> s) & 1ull))) ? 1 : 0);
+    const int np = (n + kPage - 1) / kPage;
+    pages += (long long)np * Hkv;
+    maxpages = std::max(maxpages, np);
+  }
+  // Equal page ranges for every CTA; about two CTAs per SM in total, never more than kMaxSplits per segment.
+  const int nseg = batch * Hkv, target = std::max(1, 2 * c->sm_count - nseg);
+  int pps = (int)std::max<long long>(kAttendMinPages, (pages + target - 1) / target);
+  pps = std::max(pps, (maxpages + kMaxSplits - 1) / kMaxSplits);
+  pps = std::max(1, std::min(pps, std::max(1, maxpages)));
+  const int splits = std::max(1, (maxpages + pps - 1) / pps);
+  if (scale == 0.f) scale = 1.f / sqrtf((float)D);
+  AttendArgs a;
+  a.layer = layer; a.q = (const __nv_bfloat16 *)q; a.out = (__nv_bfloat16 *)out;
+  a.scale_log2 = scale * 1.4426950408889634f; a.pps = pps; a.nst = kAttendStages; a.append = app ? 1 : 0;
+  a.k_new = (const uint8_t *)k_new; a.v_new = (const uint8_t *)v_new; a.pos_new = pos; a.seq_mask = seq_mask;
+  const int rc = D == 128 ? launch_attend_t<128>(c, a, splits, pdl, st) : launch_attend_t<64>(c, a, splits, pdl, st);
+  if (rc) return rc;
+  if (app)
+    for (int s = 0; s < batch; ++s)
+      if (!seq_mask || ((seq_mask >> s) & 1ull)) ++c->h_len[(size_t)layer * batch + s];
   return FKV_OK;
 }
 
@@ -221,6 +264,7 @@ int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, voi
   x.scores = (float *)(ws + L.scores); x.idx = (int *)(ws + L.idx); x.plan = (SegPlan *)(ws + L.plan);
   x.work = (int *)(ws + L.work); x.tile1_start = (int *)(ws + L.tile1); x.part_o = (float *)(ws + L.part_o);
   x.part_ml = (float *)(ws + L.part_ml); x.tickets = (int *)(ws + L.tickets);
+  x.seq_tickets = (int *)(ws + L.seq_tickets);
   c->h_len.assign((size_t)cfg->num_layers * cfg->max_batch, 0);
   c->h_budget.assign(cfg->max_batch, cfg->budget);
   c->loaded.assign((size_t)cfg->num_layers * cfg->num_kv_heads, 0);
@@ -407,28 +451,34 @@ int fkv_evict(fkv_cache *c, int layer, void *stream) {
 
 int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream) {
   if (!c || !layer_ok(c, layer) || !q || !out) return FKV_ERR_INVALID_ARG;
-  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads, D = c->cfg.head_dim;
-  int maxn = 0;
-  for (int s = 0; s < batch; ++s) maxn = std::max(maxn, c->h_len[(size_t)layer * batch + s]);
-  const int maxpages = (maxn + kPage - 1) / kPage;
-  int splits = (2 * c->sm_count + batch * Hkv - 1) / (batch * Hkv);
-  splits = std::max(1, std::min({splits, kMaxSplits, (maxpages + kAttendMinPages - 1) / kAttendMinPages}));
-  if (scale == 0.f) scale = 1.f / sqrtf((float)D);
-  const float scale_log2 = scale * 1.4426950408889634f;
-  cudaStream_t st = (cudaStream_t)stream;
-  return D == 128 ? launch_attend<128>(c, layer, q, out, scale_log2, splits, st)
-                  : launch_attend<64>(c, layer, q, out, scale_log2, splits, st);
+  return launch_attend(c, layer, q, out, scale, nullptr, nullptr, nullptr, 0, false, (cudaStream_t)stream);
+}
+
+int fkv_append_decode_attn(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, uint64_t seq_mask,
+                           const void *q, void *out, float scale, void *stream) {
+  if (!c || !layer_ok(c, layer) || !k || !v || !q || !out) return FKV_ERR_INVALID_ARG;
+  const int batch = c->cfg.max_batch;
+  for (int s = 0; s < batch; ++s)
+    if ((!seq_mask || ((seq_mask >> s) & 1ull)) && c->h_len[(size_t)layer * batch + s] >= c->lay.cap)
+      return FKV_ERR_CAPACITY;
+  return launch_attend(c, layer, q, out, scale, k, v, pos, seq_mask, false, (cudaStream_t)stream);
 }
 
 int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *pos, const void *q, void *out,
                     float scale, void *stream) {
   if (!c || !k || !v || !q || !out) return FKV_ERR_INVALID_ARG;
-  const size_t kv_stride = (size_t)c->cfg.max_batch * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
+  const int batch = c->cfg.max_batch;
+  for (int l = 0; l < c->cfg.num_layers; ++l)
+    for (int s = 0; s < batch; ++s)
+      if (c->h_len[(size_t)l * batch + s] >= c->lay.cap) return FKV_ERR_CAPACITY;
+  const size_t kv_stride = (size_t)batch * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
   const size_t q_stride = kv_stride * c->cfg.group_size;
   for (int l = 0; l < c->cfg.num_layers; ++l) {
-    int rc = fkv_append(c, l, (const uint8_t *)k + l * kv_stride, (const uint8_t *)v + l * kv_stride, pos, 0, stream);
-    if (rc) return rc;
-    rc = fkv_decode_attn(c, l, (const uint8_t *)q + l * q_stride, (uint8_t *)out + l * q_stride, scale, stream);
+    // Layer l's launch may start while layer l - 1's is finishing: the part of it that runs early touches
+    // only layer l's own cache state, which layer l - 1's launch does not write.
+    const int rc = launch_attend(c, l, (const uint8_t *)q + l * q_stride, (uint8_t *)out + l * q_stride, scale,
+                                 (const uint8_t *)k + l * kv_stride, (const uint8_t *)v + l * kv_stride, pos, 0, l > 0,
+                                 (cudaStream_t)stream);
     if (rc) return rc;
   }
   return FKV_OK;

@@ -62,6 +62,7 @@ struct Ctx {
   float *part_o;     // [batch*Hkv][kMaxSplits][8][D]
   float *part_ml;    // [batch*Hkv][kMaxSplits][8][2]
   int *tickets;      // [batch*Hkv]
+  int *seq_tickets;  // [batch]
 };
 
 __device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head) {
@@ -136,6 +137,35 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// ---------------------------------------------------------------- row movers
+// One warp moves one pair (K row, V row, feature row, position) between a
+// dense row and a slot of a page record.  DIR 0: dense -> page, 1: page -> dense.
+template <int DIR>
+__device__ __forceinline__ void move_row(const Ctx &c, uint8_t *page, int r, uint8_t *k, uint8_t *v, float *feat,
+                                         int32_t *pos, int lane, int32_t pos_default) {
+  const int nch = c.D >> 3;  // 16-byte chunks per K (or V) row
+  for (int q = lane; q < 2 * nch; q += 32) {
+    const int isv = q >= nch, ch = isv ? q - nch : q;
+    uint4 *pp = reinterpret_cast<uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(r, ch));
+    uint8_t *dense = isv ? v : k;
+    if (DIR == 0) {
+      *pp = dense ? *reinterpret_cast<const uint4 *>(dense + ch * 16) : make_uint4(0, 0, 0, 0);
+    } else if (dense) {
+      *reinterpret_cast<uint4 *>(dense + ch * 16) = *pp;
+    }
+  }
+  float *pf = reinterpret_cast<float *>(page + c.off_f) + r * c.F;
+  for (int f = lane; f < c.F; f += 32) {
+    if (DIR == 0) pf[f] = feat ? feat[f] : 0.f;
+    else if (feat) feat[f] = pf[f];
+  }
+  if (lane == 0) {
+    int32_t *pp = reinterpret_cast<int32_t *>(page + c.off_p) + r;
+    if (DIR == 0) *pp = pos ? *pos : pos_default;
+    else if (pos) *pos = *pp;
+  }
 }
 
 // Block-wide exclusive prefix sum of one int per thread (blockDim.x <= 1024,

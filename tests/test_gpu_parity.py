@@ -296,6 +296,73 @@ def test_attention_empty_sequence_gives_zeros():
     assert torch.all(out[0] == 0) and torch.all(torch.isfinite(out[1].float()))
 
 
+# ------------------------------------------------------------------ append + attention in one launch
+@pytest.mark.parametrize("n0", [0, 1, 15, 16, 31, 1000, 4090])
+@pytest.mark.parametrize("g,D", [(4, 128), (7, 128), (4, 64)])
+def test_fused_append_attention(n0, g, D):
+    # 36 tokens, each appended and attended by ONE launch, crossing page boundaries (and opening the
+    # very first page when the sequence starts empty); sequence 1 is shorter than sequence 0.
+    Hkv, steps = 2, 36
+    lens = (n0, n0 // 2)
+    w = wl.Workload("fused", 1, Hkv, g, D, tuple(max(1, n) for n in lens), (1 << 20,) * 2, 0, 23, "normal")
+    c = binding.from_workload(w)
+    hist = {}
+    for s in range(2):
+        K, V, A, pos = wl.layer_inputs(w, 0, s)
+        if lens[s] > 0:
+            c.prefill(0, s, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
+        for h in range(Hkv):
+            hist[(s, h)] = [bits(K)[h][:lens[s]], bits(V)[h][:lens[s]]]
+    worst = 0.0
+    for step in range(steps):
+        k, v = wl.new_kv(w, 0, step)
+        q = wl.queries(w, 0, step)
+        out = c.append_decode_attn(0, k.cuda(), v.cuda(), q.cuda())
+        ob, qb, kb, vb = bits(out), bits(q), bits(k), bits(v)
+        assert c.lengths(0) == [lens[0] + step + 1, lens[1] + step + 1]
+        for (s, h), hv in hist.items():
+            hv[0] = np.concatenate([hv[0], kb[s, h][None]]); hv[1] = np.concatenate([hv[1], vb[s, h][None]])
+            ref, ref64 = oracle.attend(qb[s, h * g:(h + 1) * g], hv[0], hv[1])
+            err = np.abs(bits_to_f64(ob[s, h * g:(h + 1) * g]) - bits_to_f64(ref))
+            worst = max(worst, float((err / np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64))).max()))
+    assert worst <= 1.0
+    for (s, h), hv in hist.items():   # the rows are in the cache, positions continue
+        k2, v2, a2, p2 = c.export_head(0, s, h)
+        assert np.array_equal(bits(k2), hv[0]) and np.array_equal(bits(v2), hv[1])
+        assert npf(p2).tolist() == list(range(lens[s] + steps))
+        assert np.all(npf(a2)[lens[s]:] == 0)
+    assert c.device_status()[0] == 0
+
+
+def test_fused_append_mask_and_decode_step_match_separate_calls():
+    # The fused launch (with a sequence mask) and the all-layer decode step give what
+    # fkv_append followed by fkv_decode_attn gives, bit for bit.
+    w = wl.Workload("fusedm", 3, 2, 4, 128, (100, 47, 16), (1 << 20,) * 3, 0, 24, "normal")
+    a, b = Loaded(w), Loaded(w)
+    for step in range(20):
+        ks = torch.stack([wl.new_kv(w, l, step)[0] for l in range(3)]).cuda()
+        vs = torch.stack([wl.new_kv(w, l, step)[1] for l in range(3)]).cuda()
+        qs = torch.stack([wl.queries(w, l, step) for l in range(3)]).cuda()
+        if step % 2 == 0:
+            out_a = a.cache.decode_step(ks, vs, qs)
+            mask = 0
+        else:
+            mask = 0b101
+            out_a = torch.stack([a.cache.append_decode_attn(l, ks[l], vs[l], qs[l], seq_mask=mask) for l in range(3)])
+        outs = []
+        for l in range(3):
+            b.cache.append(l, ks[l], vs[l], seq_mask=mask)
+            outs.append(b.cache.decode_attn(l, qs[l]))
+        assert torch.equal(out_a, torch.stack(outs))
+        assert [a.cache.lengths(l) for l in range(3)] == [b.cache.lengths(l) for l in range(3)]
+    for l in range(3):
+        for s in range(3):
+            for h in range(2):
+                for x, y in zip(a.export(l, s, h), b.export(l, s, h)):
+                    assert np.array_equal(x, y)
+    assert a.cache.device_status()[0] == 0 and b.cache.device_status()[0] == 0
+
+
 # ------------------------------------------------------------------ the decode protocol of Section 3.1
 def test_decode_schedule_sawtooth():
     # cache at B, then L appended tokens -> B + L -> evict back to B, keeping the last L (R = L).
