@@ -163,10 +163,12 @@ int fkv_append_decode_attn(fkv_cache *c, int layer, const void *k, const void *v
  * fkv_append_decode_attn(k[l], v[l], q[l]) -> out[l].  k, v: dev
  * [L][max_batch][Hkv][D] bf16; q, out: dev [L][max_batch][Hkv*g][D] bf16; pos:
  * dev [max_batch] or NULL (as fkv_append).  One launch per layer, issued from
- * native code; layer l's launch is allowed to start reading its own cache
- * while layer l-1's launch is finishing (programmatic dependent launch; q, k,
- * v and out of layer l are touched only after layer l-1's launch is complete).
- * For engines that have all layers' tensors at hand, and for benchmarks of the
+ * native code.  Every layer's k, v and q must be complete when the call is
+ * enqueued: the layers do not depend on one another here, so the launches of
+ * layers 1 .. L-1 are allowed to run alongside the launch before them
+ * (programmatic dependent launch), and out[l] is complete only when the whole
+ * step is (the next work on the stream is ordered after all of it).  For
+ * engines that have all layers' tensors at hand, and for benchmarks of the
  * attention side alone.
  */
 int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *pos, const void *q, void *out,

@@ -27,16 +27,13 @@ namespace {
 thread_local std::string g_cuda_error;
 
 constexpr int kScorePPS = 8;
-constexpr int kAttendPPS = 4;
-constexpr int kAttendStages = 3;
 constexpr int kAttendMinPages = 4;
 constexpr size_t kMaxSmem = 227 * 1024;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, part_o, part_ml,
-      tickets, seq_tickets, total;
+  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, total;
   int cap, max_pages, num_pages, page_bytes, F, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
 };
 
@@ -85,11 +82,7 @@ Layout make_layout(const fkv_config &c) {
   L.plan = take(nseg * sizeof(SegPlan));
   L.work = take(nseg * 4);
   L.tile1 = take((nseg + 1) * 4);
-  const size_t lsegs = (size_t)c.max_batch * c.num_kv_heads;
-  L.part_o = take(lsegs * kMaxSplits * 8 * D * 4);
-  L.part_ml = take(lsegs * kMaxSplits * 8 * 2 * 4);
-  L.tickets = take(lsegs * 4);
-  L.seq_tickets = take((size_t)c.max_batch * 4);
+  L.seq_tickets = take((size_t)c.num_layers * c.max_batch * 4);
   L.total = off;
   return L;
 }
@@ -114,6 +107,7 @@ struct fkv_cache {
   std::vector<uint8_t> staging;
   uint64_t launches = 0;
   int sm_count = 148;
+  int max_cluster = 0;  // largest attention cluster this device places (found at the first launch)
   bool timing = false, timed = false;
   cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
 };
@@ -173,29 +167,47 @@ int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, 
   return FKV_OK;
 }
 
-// One launch of the attention kernel for `layer`: optional fused append, optional overlap of its prologue with
-// the previous launch (pdl; only when that launch is known to be this kernel on ANOTHER layer).
-template <int D>
-int launch_attend_t(fkv_cache *c, const AttendArgs &a, int splits, bool pdl, cudaStream_t st) {
-  const size_t smem = AttendSmem::bytes(D, kAttendPPS, kAttendStages);
-  static bool attr_done = false;
-  if (!attr_done) {
-    FKV_CUDA(cudaFuncSetAttribute(k_attend<D, kAttendPPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_done = true;
-  }
+// One launch of the attention kernel: the `splits` CTAs of a segment are one cluster.  a == nullptr does the
+// once-per-handle set-up instead.  pdl: the launch may run alongside the one before it on the stream.
+template <int D, int NCW, int SLOTS>
+int launch_attend_t(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cudaStream_t st) {
+  const size_t smem = AttendSmem::bytes(D, NCW, SLOTS);
+  auto kern = k_attend<D, NCW, SLOTS>;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(splits, c->cfg.max_batch * c->cfg.num_kv_heads);
-  cfg.blockDim = dim3((kAttendPPS + 1) * 32);
+  cfg.blockDim = dim3((NCW + 1) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = pdl ? 1 : 0;
-  FKV_CUDA(cudaLaunchKernelEx(&cfg, k_attend<D, kAttendPPS>, c->ctx, a));
+  if (!a) {
+    // Opt in to the shared memory and to clusters of 16, and find the largest cluster (16, else 8) this
+    // device can actually place.
+    FKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    FKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    cfg.gridDim = dim3(16, 1);
+    at[0].val.clusterDim.x = 16;
+    cfg.numAttrs = 1;
+    int nclusters = 0;
+    const bool ok16 = cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg) == cudaSuccess && nclusters > 0;
+    (void)cudaGetLastError();
+    c->max_cluster = ok16 ? 16 : 8;
+    return FKV_OK;
+  }
+  cfg.gridDim = dim3(splits, c->cfg.max_batch * c->cfg.num_kv_heads);
+  at[0].val.clusterDim.x = splits;
+  cfg.numAttrs = pdl ? 2 : 1;
+  FKV_CUDA(cudaLaunchKernelEx(&cfg, kern, c->ctx, *a));
   ++c->launches;
   return FKV_OK;
+}
+
+int attend_dispatch(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cudaStream_t st) {
+  return c->cfg.head_dim == 128 ? launch_attend_t<128, 6, 12>(c, a, splits, pdl, st)
+                                : launch_attend_t<64, 8, 24>(c, a, splits, pdl, st);
 }
 
 // Attention over `layer`, with the new pair of every participating sequence appended first when k_new is given.
@@ -203,26 +215,28 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
                   const int32_t *pos, uint64_t seq_mask, bool pdl, cudaStream_t st) {
   const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads, D = c->cfg.head_dim;
   const bool app = k_new != nullptr;
-  long long pages = 0;
   int maxpages = 0;
   for (int s = 0; s < batch; ++s) {
     const int n = c->h_len[(size_t)layer * batch + s] + ((app && (!seq_mask || ((seq_mask >> s) & 1ull))) ? 1 : 0);
-    const int np = (n + kPage - 1) / kPage;
-    pages += (long long)np * Hkv;
-    maxpages = std::max(maxpages, np);
+    maxpages = std::max(maxpages, (n + kPage - 1) / kPage);
   }
-  // Equal page ranges for every CTA; about two CTAs per SM in total, never more than kMaxSplits per segment.
-  const int nseg = batch * Hkv, target = std::max(1, 2 * c->sm_count - nseg);
-  int pps = (int)std::max<long long>(kAttendMinPages, (pages + target - 1) / target);
-  pps = std::max(pps, (maxpages + kMaxSplits - 1) / kMaxSplits);
-  pps = std::max(1, std::min(pps, std::max(1, maxpages)));
-  const int splits = std::max(1, (maxpages + pps - 1) / pps);
+  if (c->max_cluster == 0) {
+    const int rc = attend_dispatch(c, nullptr, 0, false, st);
+    if (rc) return rc;
+  }
+  // Splits per segment: a power of two, about two CTAs per SM in total, at least kAttendMinPages pages each.
+  const int nseg = batch * Hkv, cap = std::min(c->max_cluster, kMaxSplits);
+  int splits = 1;
+  while (splits * 2 <= cap && splits * 2 * nseg <= 2 * c->sm_count &&
+         (maxpages + splits * 2 - 1) / (splits * 2) >= kAttendMinPages)
+    splits *= 2;
+  const int pps = std::max(1, (maxpages + splits - 1) / splits);
   if (scale == 0.f) scale = 1.f / sqrtf((float)D);
   AttendArgs a;
   a.layer = layer; a.q = (const __nv_bfloat16 *)q; a.out = (__nv_bfloat16 *)out;
-  a.scale_log2 = scale * 1.4426950408889634f; a.pps = pps; a.nst = kAttendStages; a.append = app ? 1 : 0;
+  a.scale_log2 = scale * 1.4426950408889634f; a.pps = pps; a.append = app ? 1 : 0;
   a.k_new = (const uint8_t *)k_new; a.v_new = (const uint8_t *)v_new; a.pos_new = pos; a.seq_mask = seq_mask;
-  const int rc = D == 128 ? launch_attend_t<128>(c, a, splits, pdl, st) : launch_attend_t<64>(c, a, splits, pdl, st);
+  const int rc = attend_dispatch(c, &a, splits, pdl, st);
   if (rc) return rc;
   if (app)
     for (int s = 0; s < batch; ++s)
@@ -262,8 +276,7 @@ int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, voi
   x.planhdr = (int *)(ws + L.planhdr); x.pt = (int *)(ws + L.pt); x.pt_new = (int *)(ws + L.pt_new);
   x.len = (int *)(ws + L.len); x.budget = (int *)(ws + L.budget); x.sp = ws + L.sp;
   x.scores = (float *)(ws + L.scores); x.idx = (int *)(ws + L.idx); x.plan = (SegPlan *)(ws + L.plan);
-  x.work = (int *)(ws + L.work); x.tile1_start = (int *)(ws + L.tile1); x.part_o = (float *)(ws + L.part_o);
-  x.part_ml = (float *)(ws + L.part_ml); x.tickets = (int *)(ws + L.tickets);
+  x.work = (int *)(ws + L.work); x.tile1_start = (int *)(ws + L.tile1);
   x.seq_tickets = (int *)(ws + L.seq_tickets);
   c->h_len.assign((size_t)cfg->num_layers * cfg->max_batch, 0);
   c->h_budget.assign(cfg->max_batch, cfg->budget);
@@ -474,8 +487,8 @@ int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *p
   const size_t kv_stride = (size_t)batch * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
   const size_t q_stride = kv_stride * c->cfg.group_size;
   for (int l = 0; l < c->cfg.num_layers; ++l) {
-    // Layer l's launch may start while layer l - 1's is finishing: the part of it that runs early touches
-    // only layer l's own cache state, which layer l - 1's launch does not write.
+    // Layer l's launch may run alongside layer l - 1's: each touches only its own layer's cache state and
+    // tensors.  Layer 0's launch is ordered after everything before it on the stream, as usual.
     const int rc = launch_attend(c, l, (const uint8_t *)q + l * q_stride, (uint8_t *)out + l * q_stride, scale,
                                  (const uint8_t *)k + l * kv_stride, (const uint8_t *)v + l * kv_stride, pos, 0, l > 0,
                                  (cudaStream_t)stream);

@@ -12,8 +12,7 @@ __global__ void k_reset(Ctx c) {
   const int stride = gridDim.x * blockDim.x, t0 = blockIdx.x * blockDim.x + threadIdx.x;
   for (int i = t0; i < c.num_pages; i += stride) c.free_stack[i] = c.num_pages - 1 - i;
   for (int i = t0; i < c.L * c.batch; i += stride) c.len[i] = 0;
-  for (int i = t0; i < c.batch * c.Hkv; i += stride) c.tickets[i] = 0;
-  for (int i = t0; i < c.batch; i += stride) c.seq_tickets[i] = 0;
+  for (int i = t0; i < c.L * c.batch; i += stride) c.seq_tickets[i] = 0;
   if (t0 == 0) {
     c.ctrl[CTRL_FREE_TOP] = c.num_pages;
     c.ctrl[CTRL_STATUS] = 0;

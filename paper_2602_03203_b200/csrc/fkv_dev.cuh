@@ -10,7 +10,6 @@ namespace fkv {
 
 constexpr int kPage = 16;        // pairs per page
 constexpr int kHidden = 16;      // scorer hidden width (Section 4.1)
-constexpr int kMaxSplits = 64;   // split-K partials kept per segment
 
 // Device status bits (mirrors include/fkv.h).
 constexpr unsigned kDevPoolExhausted = 1u, kDevCapacity = 2u, kDevWaitTimeout = 4u, kDevBadIndex = 8u;
@@ -59,10 +58,7 @@ struct Ctx {
   int *work;         // work list of segment ids
   int *tile1_start;  // prefix of score tiles over the work list
   int *planhdr;
-  float *part_o;     // [batch*Hkv][kMaxSplits][8][D]
-  float *part_ml;    // [batch*Hkv][kMaxSplits][8][2]
-  int *tickets;      // [batch*Hkv]
-  int *seq_tickets;  // [batch]
+  int *seq_tickets;  // [L][batch]
 };
 
 __device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head) {
@@ -132,6 +128,13 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Transpose of an 8 x 8 tile of 16-bit values held one row-pair per lane (the mma fragment layout).
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
