@@ -88,7 +88,7 @@ class ClockSampler:
             f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
             self.path = f.name
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=f,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -288,6 +288,10 @@ def run_ours(args):
         "evict_frac_of_nominal_8TBps": value / N / NOMINAL_HBM_GBS,
         "decode_tokens_per_s": tok_s,
         "decode_attn_gbs": N * dec_bytes / (decode_ms * 1e-3) / 1e9 if T else 0.0,
+        "decode_attn_frac_of_measured_peak": dec_bytes / (decode_ms * 1e-3) / 1e9 / peak if T else 0.0,
+        "decode_us_per_layer_launch": 1e3 * decode_ms / (T * L) if T else 0.0,
+        "decode_note": "attention side only (append + GQA attention, one launch per layer, layers of a token "
+                       "overlap); no projections, MLP or sampling",
         "roofline": {"bound": "hbm", "kernel": f"k_{dom}", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": args.traffic},
         "e2e": {"value": N * eb["total"] / (e_evict * 1e-3) / 1e9, "unit": UNIT,
@@ -311,7 +315,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3)

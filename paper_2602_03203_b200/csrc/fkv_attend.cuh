@@ -171,7 +171,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
         int32_t pdef = 0;
         if (!a.pos_new && n_old > 0) {
           const uint8_t *prev = c.pool + (size_t)ptrow[(n_old - 1) / kPage] * c.page_bytes;
-          pdef = reinterpret_cast<const int32_t *>(prev + c.off_p)[(n_old - 1) % kPage] + 1;
+          pdef = reinterpret_cast<const int32_t *>(meta_row(c, prev, (n_old - 1) % kPage))[c.F] + 1;
         }
         const size_t row = (size_t)seq * c.Hkv + head;
         move_row<0>(c, c.pool + (size_t)npid * c.page_bytes, n_old % kPage, const_cast<uint8_t *>(a.k_new) + row * D * 2,

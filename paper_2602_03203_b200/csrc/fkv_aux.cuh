@@ -63,7 +63,7 @@ __global__ void k_prefill_rows(Ctx c, int layer, int seq, int n, const uint8_t *
                 feat ? const_cast<float *>(feat) + row * c.F : nullptr, pos ? const_cast<int32_t *>(pos) + i : nullptr,
                 lane, i);
   } else {
-    float *pf = reinterpret_cast<float *>(page + c.off_f) + (i % kPage) * c.F;
+    float *pf = meta_row(c, page, i % kPage);
     for (int f = lane; f < c.F; f += 32) pf[f] = feat[row * c.F + f];
   }
 }
@@ -117,7 +117,7 @@ __global__ void k_append(Ctx c, int layer, const uint8_t *k, const uint8_t *v, c
   int32_t pdef = 0;
   if (!pos && n > 0) {
     const uint8_t *prev = c.pool + (size_t)ptrow[(n - 1) / kPage] * c.page_bytes;
-    pdef = reinterpret_cast<const int32_t *>(prev + c.off_p)[(n - 1) % kPage] + 1;
+    pdef = reinterpret_cast<const int32_t *>(meta_row(c, prev, (n - 1) % kPage))[c.F] + 1;
   }
   const size_t row = (size_t)seq * c.Hkv + h;
   move_row<0>(c, c.pool + (size_t)pid * c.page_bytes, n % kPage, const_cast<uint8_t *>(k) + row * c.D * 2,

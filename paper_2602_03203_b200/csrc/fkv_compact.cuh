@@ -6,8 +6,9 @@
 // Roofline: HBM, 2 x (4D + 4F + 4) bytes per kept pair.  grid (tiles of 64
 // output rows, work list).  The CTA first resolves index and page-table
 // lookups for all its rows in one step, then every warp moves 8 rows: all
-// loads first, then all stores, 16 bytes per lane for K and V.  The 16-byte
-// chunks are re-swizzled for the new row index on the way.
+// loads first, then all stores, 16 bytes per lane for K and V and one or two
+// 32-bit words per lane for the meta row (features + position, one run).
+// The 16-byte chunks are re-swizzled for the new row index on the way.
 #pragma once
 #include "fkv_dev.cuh"
 
@@ -45,12 +46,11 @@ __global__ void __launch_bounds__(256) k_compact(Ctx c, const int32_t *idx, int 
   }
   __syncthreads();
   // Phase 2: each warp moves 8 rows; lane = one 16-byte chunk of K (0..NCH-1) or V.
-  const int FH = c.F >> 1;  // 8-byte feature chunks per row (<= 24)
+  const int MW = c.F + 1;   // words of a meta row (<= 49): lane and lane + 32
   const int isv = lane >= NCH, ch = isv ? lane - NCH : lane;
   const bool kvlane = lane < 2 * NCH;
   uint4 kv[kCompactRPW];
-  float2 ft[kCompactRPW];
-  int32_t ps[kCompactRPW];
+  uint32_t m0[kCompactRPW], m1[kCompactRPW];
   const int r0 = warp * kCompactRPW;
 #pragma unroll
   for (int u = 0; u < kCompactRPW; ++u) {
@@ -59,8 +59,9 @@ __global__ void __launch_bounds__(256) k_compact(Ctx c, const int32_t *idx, int 
     const uint8_t *page = c.pool + (size_t)(src / kPage) * c.page_bytes;
     const int sr = (int)(src % kPage);
     if (kvlane) kv[u] = *reinterpret_cast<const uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(sr, ch));
-    if (lane < FH) ft[u] = reinterpret_cast<const float2 *>(page + c.off_f)[sr * FH + lane];
-    if (lane == 31) ps[u] = reinterpret_cast<const int32_t *>(page + c.off_p)[sr];
+    const uint32_t *mr = reinterpret_cast<const uint32_t *>(meta_row(c, page, sr));
+    if (lane < MW) m0[u] = mr[lane];
+    if (lane + 32 < MW) m1[u] = mr[lane + 32];
   }
 #pragma unroll
   for (int u = 0; u < kCompactRPW; ++u) {
@@ -68,8 +69,9 @@ __global__ void __launch_bounds__(256) k_compact(Ctx c, const int32_t *idx, int 
     const int jr = r0 + u, dr = jr % kPage;
     uint8_t *page = c.pool + (size_t)s_dst[jr / kPage] * c.page_bytes;
     if (kvlane) *reinterpret_cast<uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(dr, ch)) = kv[u];
-    if (lane < FH) reinterpret_cast<float2 *>(page + c.off_f)[dr * FH + lane] = ft[u];
-    if (lane == 31) reinterpret_cast<int32_t *>(page + c.off_p)[dr] = ps[u];
+    uint32_t *mr = reinterpret_cast<uint32_t *>(meta_row(c, page, dr));
+    if (lane < MW) mr[lane] = m0[u];
+    if (lane + 32 < MW) mr[lane + 32] = m1[u];
   }
 }
 

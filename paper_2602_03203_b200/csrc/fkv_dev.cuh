@@ -31,10 +31,11 @@ struct SegPlan {
 };
 
 // One page record holds 16 pairs of one segment:
-//   K   [D/64][16][64] bf16, 16-byte chunks XOR-swizzled inside each 128-byte row
-//   V   same layout
-//   a   [16][F] fp32 attention features
-//   pos [16] int32 original token positions
+//   K    [D/64][16][64] bf16, 16-byte chunks XOR-swizzled inside each 128-byte row
+//   V    same layout
+//   meta [16][F + 1] 32-bit words: the pair's F fp32 attention features, then its
+//        original token position (int32) - one contiguous run per pair, so a
+//        gather of the pair touches one place for both
 // The swizzle (chunk c of row r sits at chunk c ^ (r & 7)) is the 128-byte
 // shared-memory swizzle, applied in HBM so that ONE bulk copy of the record
 // lands in shared memory ready for conflict-free ldmatrix.
@@ -43,7 +44,7 @@ struct Ctx {
   int cap;        // segment capacity in pairs (multiple of 16)
   int max_pages;  // cap / 16
   int num_pages;
-  int page_bytes, off_v, off_f, off_p;
+  int page_bytes, off_v, off_f;  // off_f: start of the meta rows (F + 1 words each)
   int sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
   uint8_t *pool;
   int *free_stack;
@@ -69,6 +70,14 @@ __device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head
 // (8 channels) of row `r`.
 __device__ __forceinline__ int kv_chunk_off(int r, int ch) {
   return ((ch >> 3) << 11) + (r << 7) + (((ch & 7) ^ (r & 7)) << 4);
+}
+
+// Meta row of pair r of a page record: F feature floats, then the position id.
+__device__ __forceinline__ float *meta_row(const Ctx &c, uint8_t *page, int r) {
+  return reinterpret_cast<float *>(page + c.off_f) + r * (c.F + 1);
+}
+__device__ __forceinline__ const float *meta_row(const Ctx &c, const uint8_t *page, int r) {
+  return reinterpret_cast<const float *>(page + c.off_f) + r * (c.F + 1);
 }
 
 __device__ __forceinline__ void set_status(const Ctx &c, unsigned bits) { atomicOr((unsigned *)&c.ctrl[CTRL_STATUS], bits); }
@@ -159,13 +168,13 @@ __device__ __forceinline__ void move_row(const Ctx &c, uint8_t *page, int r, uin
       *reinterpret_cast<uint4 *>(dense + ch * 16) = *pp;
     }
   }
-  float *pf = reinterpret_cast<float *>(page + c.off_f) + r * c.F;
+  float *pf = meta_row(c, page, r);
   for (int f = lane; f < c.F; f += 32) {
     if (DIR == 0) pf[f] = feat ? feat[f] : 0.f;
     else if (feat) feat[f] = pf[f];
   }
   if (lane == 0) {
-    int32_t *pp = reinterpret_cast<int32_t *>(page + c.off_p) + r;
+    int32_t *pp = reinterpret_cast<int32_t *>(pf + c.F);
     if (DIR == 0) *pp = pos ? *pos : pos_default;
     else if (pos) *pos = *pp;
   }

@@ -137,11 +137,10 @@ __global__ void __launch_bounds__((PPS + 1) * 32, 1) k_score(Ctx c, float *out, 
       }
       // Feature columns in fp32: this lane owns hidden units {2t, 2t+1, 8+2t, 9+2t} of rows gid and gid+8.
       float fz[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-      const float *f0 = reinterpret_cast<const float *>(page + c.off_f) + gid * c.F;
-      const float *f1 = f0 + 8 * c.F;
+      const float *f0 = meta_row(c, page, gid), *f1 = meta_row(c, page, gid + 8);   // odd word stride: no bank conflicts
       const float4 *wf = reinterpret_cast<const float4 *>(sp + c.sp_off_wf) + tig;
       for (int f = 0; f < c.F; f += 2) {
-        const float2 x0 = *reinterpret_cast<const float2 *>(f0 + f), x1 = *reinterpret_cast<const float2 *>(f1 + f);
+        const float2 x0 = make_float2(f0[f], f0[f + 1]), x1 = make_float2(f1[f], f1[f + 1]);
         const float4 wa = __ldg(wf + f * 4), wb = __ldg(wf + f * 4 + 4);
         fz[0][0] = fmaf(x0.x, wa.x, fz[0][0]); fz[0][1] = fmaf(x0.x, wa.y, fz[0][1]);
         fz[0][2] = fmaf(x0.x, wa.z, fz[0][2]); fz[0][3] = fmaf(x0.x, wa.w, fz[0][3]);
