@@ -98,21 +98,23 @@ __global__ void __launch_bounds__((PPS + 1) * 32, 1) k_score(Ctx c, float *out, 
   // ---------------- consumers: warp w owns page w of every stage ----------------
   const int gid = lane >> 2, tig = lane & 3;
   uint32_t bw[KS][4];  // W1 (K and V rows) as mma B fragments: both 8-wide halves of the 16 hidden units
-  int cur_sp = -1;
   const uint8_t *sp = nullptr;
+  float4 b1 = make_float4(0.f, 0.f, 0.f, 0.f), w2 = b1;
+  float b2 = 0.f;
+  // The work item this warp is in: its tiles [tbeg, tend), its segment and length.  Reloaded only on a change.
+  int tbeg = 0, tend = -1, seg = 0, n = 0;
   // ldmatrix row address pieces for this lane: matrix mi = lane / 8 covers rows (mi & 1) * 8 .. +8
   // and the low (mi < 2) or high 8 channels of a 16-channel step.
   const int lrow = ((lane >> 3) & 1) * 8 + (lane & 7), lhi = lane >> 4;
 
   for (int t = t0, it = 0; t < t1; ++t, ++it) {
     const int s = it % nst, ph = (it / nst) & 1;
-    while (t >= c.tile1_start[wi + 1]) ++wi;
-    const int seg = c.work[wi], tin = t - c.tile1_start[wi];
-    const int n = c.plan[seg].n_old;
-    const int np = min(PPS, (n + kPage - 1) / kPage - tin * PPS);
-    const int spi = (seg / (c.batch * c.Hkv)) * c.Hkv + seg % c.Hkv;  // (layer, head)
-    if (spi != cur_sp) {
-      cur_sp = spi;
+    if (t >= tend) {
+      while (t >= c.tile1_start[wi + 1]) ++wi;
+      tbeg = c.tile1_start[wi]; tend = c.tile1_start[wi + 1];
+      seg = c.work[wi];
+      n = c.plan[seg].n_old;
+      const int spi = (seg / (c.batch * c.Hkv)) * c.Hkv + seg % c.Hkv;  // (layer, head)
       sp = c.sp + (size_t)spi * c.sp_stride;
       const uint4 *w = reinterpret_cast<const uint4 *>(sp);
 #pragma unroll
@@ -120,40 +122,53 @@ __global__ void __launch_bounds__((PPS + 1) * 32, 1) k_score(Ctx c, float *out, 
         uint4 x = __ldg(w + ks * 32 + lane);
         bw[ks][0] = x.x; bw[ks][1] = x.y; bw[ks][2] = x.z; bw[ks][3] = x.w;
       }
+      b1 = __ldg(reinterpret_cast<const float4 *>(sp + c.sp_off_b1) + tig);
+      w2 = __ldg(reinterpret_cast<const float4 *>(sp + c.sp_off_w2) + tig);
+      b2 = __ldg(reinterpret_cast<const float *>(sp + c.sp_off_b2));
     }
+    const int tin = t - tbeg;
+    const int np = min(PPS, (n + kPage - 1) / kPage - tin * PPS);
     if (!mbar_wait(smem_u32(&bars[s]), ph)) { set_status(c, kDevWaitTimeout); break; }
     if (warp < np) {
       const uint8_t *page = smem + (size_t)s * stage_bytes + warp * pitch;
       const uint32_t kbase = smem_u32(page), vbase = kbase + c.off_v;
+      // Two accumulation chains per half of the hidden units (K channels and V channels), summed below
+      // in a fixed order: half the dependent-mma depth.
       float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      float acv[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        const int kk = ks % KSH;                  // 16-channel step inside K or V
-        const int ch = kk * 2 + lhi;              // 16-byte chunk this lane addresses
-        uint32_t a[4];
-        ldsm_x4(a, (ks < KSH ? kbase : vbase) + kv_chunk_off(lrow, ch));
-        mma_bf16(acc[0], a[0], a[1], a[2], a[3], bw[ks][0], bw[ks][1]);
-        mma_bf16(acc[1], a[0], a[1], a[2], a[3], bw[ks][2], bw[ks][3]);
+      for (int kk = 0; kk < KSH; ++kk) {           // 16-channel step inside K and inside V
+        const int ch = kk * 2 + lhi;               // 16-byte chunk this lane addresses
+        uint32_t a[4], b[4];
+        ldsm_x4(a, kbase + kv_chunk_off(lrow, ch));
+        ldsm_x4(b, vbase + kv_chunk_off(lrow, ch));
+        mma_bf16(acc[0], a[0], a[1], a[2], a[3], bw[kk][0], bw[kk][1]);
+        mma_bf16(acc[1], a[0], a[1], a[2], a[3], bw[kk][2], bw[kk][3]);
+        mma_bf16(acv[0], b[0], b[1], b[2], b[3], bw[KSH + kk][0], bw[KSH + kk][1]);
+        mma_bf16(acv[1], b[0], b[1], b[2], b[3], bw[KSH + kk][2], bw[KSH + kk][3]);
       }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { acc[0][i] += acv[0][i]; acc[1][i] += acv[1][i]; }
       // Feature columns in fp32: this lane owns hidden units {2t, 2t+1, 8+2t, 9+2t} of rows gid and gid+8.
       float fz[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
       const float *f0 = meta_row(c, page, gid), *f1 = meta_row(c, page, gid + 8);   // odd word stride: no bank conflicts
       const float4 *wf = reinterpret_cast<const float4 *>(sp + c.sp_off_wf) + tig;
-      for (int f = 0; f < c.F; f += 2) {
-        const float2 x0 = make_float2(f0[f], f0[f + 1]), x1 = make_float2(f1[f], f1[f + 1]);
-        const float4 wa = __ldg(wf + f * 4), wb = __ldg(wf + f * 4 + 4);
-        fz[0][0] = fmaf(x0.x, wa.x, fz[0][0]); fz[0][1] = fmaf(x0.x, wa.y, fz[0][1]);
-        fz[0][2] = fmaf(x0.x, wa.z, fz[0][2]); fz[0][3] = fmaf(x0.x, wa.w, fz[0][3]);
-        fz[1][0] = fmaf(x1.x, wa.x, fz[1][0]); fz[1][1] = fmaf(x1.x, wa.y, fz[1][1]);
-        fz[1][2] = fmaf(x1.x, wa.z, fz[1][2]); fz[1][3] = fmaf(x1.x, wa.w, fz[1][3]);
-        fz[0][0] = fmaf(x0.y, wb.x, fz[0][0]); fz[0][1] = fmaf(x0.y, wb.y, fz[0][1]);
-        fz[0][2] = fmaf(x0.y, wb.z, fz[0][2]); fz[0][3] = fmaf(x0.y, wb.w, fz[0][3]);
-        fz[1][0] = fmaf(x1.y, wb.x, fz[1][0]); fz[1][1] = fmaf(x1.y, wb.y, fz[1][1]);
-        fz[1][2] = fmaf(x1.y, wb.z, fz[1][2]); fz[1][3] = fmaf(x1.y, wb.w, fz[1][3]);
+      for (int f = 0; f < c.F; f += 6) {   // one query head's six features at a time: all loads, then the FMAs
+        float x0[6], x1[6];
+        float4 w[6];
+#pragma unroll
+        for (int j = 0; j < 6; ++j) {
+          x0[j] = f0[f + j]; x1[j] = f1[f + j];
+          w[j] = __ldg(wf + (f + j) * 4);
+        }
+#pragma unroll
+        for (int j = 0; j < 6; ++j) {
+          fz[0][0] = fmaf(x0[j], w[j].x, fz[0][0]); fz[0][1] = fmaf(x0[j], w[j].y, fz[0][1]);
+          fz[0][2] = fmaf(x0[j], w[j].z, fz[0][2]); fz[0][3] = fmaf(x0[j], w[j].w, fz[0][3]);
+          fz[1][0] = fmaf(x1[j], w[j].x, fz[1][0]); fz[1][1] = fmaf(x1[j], w[j].y, fz[1][1]);
+          fz[1][2] = fmaf(x1[j], w[j].z, fz[1][2]); fz[1][3] = fmaf(x1[j], w[j].w, fz[1][3]);
+        }
       }
-      const float4 b1 = __ldg(reinterpret_cast<const float4 *>(sp + c.sp_off_b1) + tig);
-      const float4 w2 = __ldg(reinterpret_cast<const float4 *>(sp + c.sp_off_w2) + tig);
-      const float b2 = __ldg(reinterpret_cast<const float *>(sp + c.sp_off_b2));
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
         const float z0 = acc[0][2 * r] + fz[r][0] + b1.x, z1 = acc[0][2 * r + 1] + fz[r][1] + b1.y;
