@@ -26,7 +26,7 @@ namespace {
 
 thread_local std::string g_cuda_error;
 
-constexpr int kScorePPS = 8;
+constexpr int kScorePPS = 8;  // consumer warps of the scorer = pages per tile
 constexpr int kAttendMinPages = 4;
 constexpr size_t kMaxSmem = 227 * 1024;
 
@@ -132,23 +132,25 @@ int cuda_fail(cudaError_t e) {
 
 bool layer_ok(const fkv_cache *c, int layer) { return layer >= 0 && layer < c->cfg.num_layers; }
 
-int score_stages(const fkv_cache *c) {
-  const size_t stage = (size_t)kScorePPS * ScoreSmem::pitch(c->lay.page_bytes);
-  return (int)std::max<size_t>(2, std::min<size_t>(4, (kMaxSmem - 256) / stage));
+// Page slots per consumer warp of the scorer: as many as fit the shared memory, at most 4.
+int score_slots_per_warp(const fkv_cache *c) {
+  for (int spw = 4; spw >= 1; --spw)
+    if (ScoreSmem::bytes(c->lay.page_bytes, c->lay.F, kScorePPS, spw) <= kMaxSmem) return spw;
+  return 0;
 }
 
 template <int D>
 int launch_score(fkv_cache *c, float *out, int seg_base, int tiles_bound, cudaStream_t st) {
-  const int nst = score_stages(c);
-  const size_t smem = ScoreSmem::bytes(c->lay.page_bytes, kScorePPS, nst);
-  if (smem > kMaxSmem) return FKV_ERR_INVALID_ARG;
+  const int spw = score_slots_per_warp(c);
+  if (spw == 0) return FKV_ERR_INVALID_ARG;
+  const size_t smem = ScoreSmem::bytes(c->lay.page_bytes, c->lay.F, kScorePPS, spw);
   static bool attr_done = false;
   if (!attr_done) {
     FKV_CUDA(cudaFuncSetAttribute(k_score<D, kScorePPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
     attr_done = true;
   }
   const int grid = std::max(1, std::min(c->sm_count, tiles_bound));
-  k_score<D, kScorePPS><<<grid, (kScorePPS + 1) * 32, smem, st>>>(c->ctx, out, seg_base, nst);
+  k_score<D, kScorePPS><<<grid, (kScorePPS + 1) * 32, smem, st>>>(c->ctx, out, seg_base, spw);
   FKV_LAUNCHED(c);
   return FKV_OK;
 }
