@@ -108,6 +108,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) k_score(Ctx c, float *out, 
       const int pg = (t - tbeg) * NCW + lane;
       pid = pg * kPage < n ? c.pt[(size_t)seg * c.max_pages + pg] : -1;
     };
+    const uint64_t stream_once = l2_policy_evict_first();   // every page passes through L2 exactly once here
     int pid, pid_next = -1;
     lookup(t0, pid);
     for (int t = t0; t < t1; ++t) {
@@ -116,8 +117,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) k_score(Ctx c, float *out, 
         const int slot = lane + NCW * ks;
         if (!mbar_wait(smem_u32(&bars[nslots + slot]), ph ^ 1)) { set_status(c, kDevWaitTimeout); break; }
         mbar_arrive_expect_tx(smem_u32(&bars[slot]), (uint32_t)c.page_bytes);
-        bulk_g2s(smem_u32(smem + (size_t)slot * pitch), c.pool + (size_t)pid * c.page_bytes, (uint32_t)c.page_bytes,
-                 smem_u32(&bars[slot]));
+        bulk_g2s_hint(smem_u32(smem + (size_t)slot * pitch), c.pool + (size_t)pid * c.page_bytes,
+                      (uint32_t)c.page_bytes, smem_u32(&bars[slot]), stream_once);
         if (++ks == spw) { ks = 0; ph ^= 1; }
       }
       pid = pid_next;
@@ -135,6 +136,9 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) k_score(Ctx c, float *out, 
   // and the low (mi < 2) or high 8 channels of a 16-channel step.
   const int lrow = ((lane >> 3) & 1) * 8 + (lane & 7), lhi = lane >> 4;
   int ks = 0, ph = 0;
+  // The scores are read back by the selection kernel right away: keep them in L2, so that no write
+  // goes to DRAM in the middle of the read stream.
+  const uint64_t keep = l2_policy_evict_last();
 
   for (int t = t0; t < t1; ++t) {
     if (t >= tend) {
@@ -209,12 +213,12 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) k_score(Ctx c, float *out, 
     float p[2];
     if (c.act == 0) score_rows<0>(acc, fz, b1, w2, 0, p);
     else score_rows<1>(acc, fz, b1, w2, c.act, p);
-    const int slot = tin * TILE + warp * kPage + gid;
-    if (tig == 0) {
-      float *o = out + (size_t)(seg - seg_base) * c.cap + slot;
-      if (slot < n) o[0] = p[0] + b2;
-      if (slot + 8 < n) o[8] = p[1] + b2;
-    }
+    // Every lane of a quad holds both sums; lane l < 16 takes the score of row l (from quad l % 8), so
+    // the page's sixteen scores leave as one 64-byte store.
+    const float lo = __shfl_sync(0xffffffffu, p[0], (lane & 7) * 4), hi = __shfl_sync(0xffffffffu, p[1], (lane & 7) * 4);
+    const float mine = lane < 8 ? lo : hi;
+    const int slot = tin * TILE + warp * kPage + lane;
+    if (lane < kPage && slot < n) st_f32_hint(out + (size_t)(seg - seg_base) * c.cap + slot, mine + b2, keep);
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&bars[nslots + slot_i]));
     if (++ks == spw) { ks = 0; ph ^= 1; }
