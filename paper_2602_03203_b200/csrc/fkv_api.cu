@@ -270,7 +270,7 @@ int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, voi
   x.L = cfg->num_layers; x.Hkv = cfg->num_kv_heads; x.G = cfg->group_size; x.D = cfg->head_dim;
   x.batch = cfg->max_batch; x.act = cfg->activation; x.R = cfg->recent_keep; x.F = L.F;
   x.cap = L.cap; x.max_pages = L.max_pages; x.num_pages = L.num_pages;
-  x.page_bytes = L.page_bytes; x.off_v = 32 * cfg->head_dim; x.off_f = 64 * cfg->head_dim;
+  x.page_bytes = L.page_bytes; x.off_v = 2 * cfg->head_dim; x.off_f = 64 * cfg->head_dim;
   x.sp_stride = L.sp_stride; x.sp_off_wf = L.sp_off_wf; x.sp_off_b1 = L.sp_off_b1; x.sp_off_w2 = L.sp_off_w2;
   x.sp_off_b2 = L.sp_off_b2;
   x.pool = ws + L.pool; x.free_stack = (int *)(ws + L.free_stack); x.ctrl = (int *)(ws + L.ctrl);

@@ -222,18 +222,18 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
           __syncwarp();
         }
         if (lane < 2 * NCH)
-          *reinterpret_cast<uint4 *>(page + (lane < NCH ? 0 : 2 * D * kPage) + kv_chunk_off(n_old % kPage, lane % NCH)) =
+          *reinterpret_cast<uint4 *>(page + (lane < NCH ? 0 : 2 * D) + kv_chunk_off(n_old % kPage, lane % NCH, D)) =
               newrow;
         __syncwarp();
       }
-      const uint32_t kbase = smem_u32(page), vbase = kbase + 2 * D * kPage;
+      const uint32_t kbase = smem_u32(page), vbase = kbase + 2 * D;
       // S^T (16 keys x 8 queries) = K (16 x D) Q^T (D x 8): keys on the M axis, two accumulation chains.
       float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int ks = 0; ks < KSQ; ks += 2) {
         uint32_t x[4], z[4];
-        ldsm_x4(x, kbase + kv_chunk_off(krow, ks * 2 + khi));
-        ldsm_x4(z, kbase + kv_chunk_off(krow, ks * 2 + 2 + khi));
+        ldsm_x4(x, kbase + kv_chunk_off(krow, ks * 2 + khi, D));
+        ldsm_x4(z, kbase + kv_chunk_off(krow, ks * 2 + 2 + khi, D));
         mma_bf16(sa, x[0], x[1], x[2], x[3], qb[ks][0], qb[ks][1]);
         mma_bf16(sb, z[0], z[1], z[2], z[3], qb[ks + 1][0], qb[ks + 1][1]);
       }
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
         uint32_t x[4];
-        ldsm_x4_trans(x, vbase + kv_chunk_off(vrow, mt * 2 + vhi));
+        ldsm_x4_trans(x, vbase + kv_chunk_off(vrow, mt * 2 + vhi, D));
         o[mt][0] *= c0; o[mt][1] *= c1; o[mt][2] *= c0; o[mt][3] *= c1;
         mma_bf16(o[mt], x[0], x[1], x[2], x[3], pb0, pb1);
       }

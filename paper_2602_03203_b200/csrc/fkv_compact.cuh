@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(256) k_compact(Ctx c, const int32_t *idx, int 
     if (src < 0) continue;
     const uint8_t *page = c.pool + (size_t)(src / kPage) * c.page_bytes;
     const int sr = (int)(src % kPage);
-    if (kvlane) kv[u] = *reinterpret_cast<const uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(sr, ch));
+    if (kvlane) kv[u] = *reinterpret_cast<const uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(sr, ch, D));
     const uint32_t *mr = reinterpret_cast<const uint32_t *>(meta_row(c, page, sr));
     if (lane < MW) m0[u] = mr[lane];
     if (lane + 32 < MW) m1[u] = mr[lane + 32];
@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(256) k_compact(Ctx c, const int32_t *idx, int 
     if (s_src[r0 + u] < 0) continue;
     const int jr = r0 + u, dr = jr % kPage;
     uint8_t *page = c.pool + (size_t)s_dst[jr / kPage] * c.page_bytes;
-    if (kvlane) *reinterpret_cast<uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(dr, ch)) = kv[u];
+    if (kvlane) *reinterpret_cast<uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(dr, ch, D)) = kv[u];
     uint32_t *mr = reinterpret_cast<uint32_t *>(meta_row(c, page, dr));
     if (lane < MW) mr[lane] = m0[u];
     if (lane + 32 < MW) mr[lane + 32] = m1[u];

@@ -31,14 +31,16 @@ struct SegPlan {
 };
 
 // One page record holds 16 pairs of one segment:
-//   K    [D/64][16][64] bf16, 16-byte chunks XOR-swizzled inside each 128-byte row
-//   V    same layout
+//   kv   [16][K row (D bf16) | V row (D bf16)]: a pair's key and value are one contiguous 4D-byte run
+//        (a gather of the pair reads one place); the 16-byte chunks of every 128-byte span are
+//        XOR-swizzled by the row index
 //   meta [16][F + 1] 32-bit words: the pair's F fp32 attention features, then its
 //        original token position (int32) - one contiguous run per pair, so a
 //        gather of the pair touches one place for both
 // The swizzle (chunk c of row r sits at chunk c ^ (r & 7)) is the 128-byte
 // shared-memory swizzle, applied in HBM so that ONE bulk copy of the record
-// lands in shared memory ready for conflict-free ldmatrix.
+// lands in shared memory ready for conflict-free ldmatrix (rows are a
+// multiple of 128 bytes apart).
 struct Ctx {
   int L, Hkv, G, D, batch, act, R, F;
   int cap;        // segment capacity in pairs (multiple of 16)
@@ -66,10 +68,10 @@ __device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head
   return (layer * c.batch + seq) * c.Hkv + head;
 }
 
-// Byte offset, inside the K (or V) part of a page record, of 16-byte chunk `ch`
-// (8 channels) of row `r`.
-__device__ __forceinline__ int kv_chunk_off(int r, int ch) {
-  return ((ch >> 3) << 11) + (r << 7) + (((ch & 7) ^ (r & 7)) << 4);
+// Byte offset, inside a page record, of 16-byte chunk `ch` (8 channels) of the K row of pair r; the V row
+// follows the K row (+ 2D bytes).  Chunks are XOR-swizzled by the row index inside each 128-byte span.
+__device__ __forceinline__ int kv_chunk_off(int r, int ch, int D) {
+  return r * (4 * D) + ((ch >> 3) << 7) + (((ch & 7) ^ (r & 7)) << 4);
 }
 
 // Meta row of pair r of a page record: F feature floats, then the position id.
@@ -182,7 +184,7 @@ __device__ __forceinline__ void move_row(const Ctx &c, uint8_t *page, int r, uin
   const int nch = c.D >> 3;  // 16-byte chunks per K (or V) row
   for (int q = lane; q < 2 * nch; q += 32) {
     const int isv = q >= nch, ch = isv ? q - nch : q;
-    uint4 *pp = reinterpret_cast<uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(r, ch));
+    uint4 *pp = reinterpret_cast<uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(r, ch, c.D));
     uint8_t *dense = isv ? v : k;
     if (DIR == 0) {
       *pp = dense ? *reinterpret_cast<const uint4 *>(dense + ch * 16) : make_uint4(0, 0, 0, 0);

@@ -179,8 +179,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) k_score(Ctx c, float *out, 
     for (int kk = 0; kk < KSH; ++kk) {           // 16-channel step inside K and inside V
       const int ch = kk * 2 + lhi;               // 16-byte chunk this lane addresses
       uint32_t a[4], b[4];
-      ldsm_x4(a, kbase + kv_chunk_off(lrow, ch));
-      ldsm_x4(b, vbase + kv_chunk_off(lrow, ch));
+      ldsm_x4(a, kbase + kv_chunk_off(lrow, ch, D));
+      ldsm_x4(b, vbase + kv_chunk_off(lrow, ch, D));
       mma_bf16(ac[kk & 1][0], a[0], a[1], a[2], a[3], bw[kk][0], bw[kk][1]);
       mma_bf16(ac[kk & 1][1], a[0], a[1], a[2], a[3], bw[kk][2], bw[kk][3]);
       mma_bf16(ac[2 + (kk & 1)][0], b[0], b[1], b[2], b[3], bw[KSH + kk][0], bw[KSH + kk][1]);
