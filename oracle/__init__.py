@@ -74,6 +74,25 @@ def select(phi, B, R=0):
     return kept[:nk].copy()
 
 
+def select_sampled(phi, B, R, noise):
+    """Sampled eviction action: kept slots (ascending int32) and the candidate slots (slot order).
+
+    noise: standard Gumbel draws, one per candidate in slot order (at least min(2 (n - B), n - r) of them).
+    """
+    phi, pphi = _c(phi, np.float32)
+    noise, pnoise = _c(noise, np.float32)
+    n = phi.shape[0]
+    kept = np.empty(max(1, min(B, n)), np.int32)
+    cand = np.empty(max(1, n), np.int32)
+    ncand = ctypes.c_int32(0)
+    need = 0 if n <= B else min(2 * (n - B), n - min(R, B))
+    assert noise.shape[0] >= need, (noise.shape, need)
+    lib().fkv_oracle_select_sampled.restype = ctypes.c_int
+    nk = lib().fkv_oracle_select_sampled(pphi, n, int(B), int(R), pnoise, kept.ctypes.data_as(ctypes.c_void_p),
+                                         cand.ctypes.data_as(ctypes.c_void_p), ctypes.byref(ncand))
+    return kept[:nk].copy(), cand[:ncand.value].copy()
+
+
 def compact(K, V, A, pos, kept):
     K, pK = _c(K, np.uint16)
     V, pV = _c(V, np.uint16)

@@ -124,6 +124,60 @@ int fkv_oracle_select(const float *phi, int n, int B, int R, int32_t *kept) {
   return B;
 }
 
+/* Lower score first; equal scores: HIGHER slot first (the order in which the deterministic rule gives pairs up). */
+static int by_score_asc_then_slot_desc(const void *pa, const void *pb) { return -by_score_then_slot(pa, pb); }
+
+/*
+ * Sampled eviction action (Section 3.1, second equation; Appendix B.2):
+ *   D = Multinomial_E( Softmax( Top_2E(-Phi) ) ),  s' = s \ D,
+ * with E = n - B pairs to evict (the paper's L).  Steps, in the paper's order:
+ *   (i)  candidates: the 2E competing pairs with the LOWEST scores (all of them if fewer compete);
+ *   (ii) p = softmax(-phi) over the candidates, then E draws without replacement.
+ * The draws are made with caller-supplied standard Gumbel noise g_j, one value per candidate in
+ * slot order (rank j): drawing without replacement from softmax(l) is the same as taking the E
+ * largest l_j + g_j (Gumbel-top-k), so with l_j = -phi_j the evicted candidates are the E with
+ * the largest (-phi_j + g_j); the softmax's normaliser cancels.  That sum is taken in fp32, the
+ * precision the decision is made in.  Ties: the higher slot is evicted.  NaN counts as -infinity,
+ * -0 as +0, both for the candidate ranking and for the perturbed value.
+ * Writes the kept slots (ascending, then the protected recent ones) and returns their number.
+ * cand_out (may be NULL, room for min(2E, n - r)) receives the candidate slots in slot order.
+ */
+int fkv_oracle_select_sampled(const float *phi, int n, int B, int R, const float *noise, int32_t *kept,
+                              int32_t *cand_out, int32_t *ncand_out) {
+  if (ncand_out) *ncand_out = 0;
+  if (n <= B) {
+    for (int i = 0; i < n; ++i) kept[i] = i;
+    return n;
+  }
+  int r = R < B ? R : B;
+  int m = n - r;                 /* pairs that compete */
+  int E = n - B;                 /* pairs to evict */
+  int C = 2 * E < m ? 2 * E : m; /* candidates */
+  ranked_t *order = (ranked_t *)malloc((size_t)m * sizeof(ranked_t));
+  for (int i = 0; i < m; ++i) { order[i].score = canonical(phi[i]); order[i].slot = i; }
+  qsort(order, (size_t)m, sizeof(ranked_t), by_score_asc_then_slot_desc);
+  int32_t *cand = (int32_t *)malloc((size_t)C * sizeof(int32_t));
+  for (int j = 0; j < C; ++j) cand[j] = order[j].slot;
+  qsort(cand, (size_t)C, sizeof(int32_t), by_slot);
+  if (cand_out) memcpy(cand_out, cand, (size_t)C * sizeof(int32_t));
+  if (ncand_out) *ncand_out = C;
+  /* perturbed logit of candidate j; rank by it, largest first, ties: higher slot first */
+  ranked_t *pert = (ranked_t *)malloc((size_t)C * sizeof(ranked_t));
+  for (int j = 0; j < C; ++j) {
+    float keep_priority = phi[cand[j]] - noise[j];          /* = -(-phi + g), one fp32 subtraction */
+    pert[j].score = canonical(keep_priority);
+    pert[j].slot = cand[j];
+  }
+  qsort(pert, (size_t)C, sizeof(ranked_t), by_score_asc_then_slot_desc);   /* lowest keep-priority = largest -phi+g */
+  char *evicted = (char *)calloc((size_t)m, 1);
+  for (int j = 0; j < E; ++j) evicted[pert[j].slot] = 1;
+  int k = 0;
+  for (int i = 0; i < m; ++i) if (!evicted[i]) kept[k++] = i;
+  for (int j = 0; j < r; ++j) kept[k + j] = m + j;
+  free(order); free(cand); free(pert); free(evicted);
+  return B;
+}
+
 /* Compaction (s' = s \ D): row j of the output is row kept[j] of the input. */
 void fkv_oracle_compact(const uint16_t *K, const uint16_t *V, const float *A, const int32_t *pos, int D, int F,
                         const int32_t *kept, int nk, uint16_t *K2, uint16_t *V2, float *A2, int32_t *pos2) {

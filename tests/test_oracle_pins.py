@@ -292,3 +292,89 @@ def test_batch_drivers_equal_single_segment_calls():
     for i in range(len(ns)):
         o = int(off[i])
         assert np.array_equal(out[i], oracle.attend(qs[i], K2[o:o + nkept[i]], V2[o:o + nkept[i]])[0])
+
+
+# ---------------------------------------------------------------- sampled eviction action (Section 3.1, Eq. 2; App. B.2)
+def _random_scores(rng, n, kind):
+    x = rng.standard_normal(n).astype(np.float32)
+    if kind == "ties":
+        x = (np.round(x * 3) / 3).astype(np.float32)
+    if kind == "special":
+        for val in (np.nan, -0.0, 0.0, np.inf, -np.inf):
+            x[rng.integers(0, n, max(1, n // 20))] = val
+    return x
+
+
+@pytest.mark.parametrize("kind", ["normal", "ties", "special"])
+def test_sampled_zero_noise_is_the_deterministic_rule(kind):
+    # With no perturbation the E largest -phi among the candidates are the E lowest scores:
+    # the action reduces to plain Top-K (the ablation's "Top-K" row), which is pinned above.
+    rng = np.random.default_rng(5)
+    for _ in range(60):
+        n = int(rng.integers(2, 300)); B = int(rng.integers(1, n + 2)); R = int(rng.integers(0, 40))
+        phi = _random_scores(rng, n, kind)
+        kept, cand = oracle.select_sampled(phi, B, R, np.zeros(2 * n, np.float32))
+        assert np.array_equal(kept, oracle.select(phi, B, R))
+
+
+def test_sampled_invariants_and_candidate_set():
+    rng = np.random.default_rng(6)
+    for _ in range(100):
+        n = int(rng.integers(3, 400)); B = int(rng.integers(1, n)); R = int(rng.integers(0, 30))
+        phi = _random_scores(rng, n, "ties" if _ % 2 else "normal")
+        noise = rng.gumbel(size=2 * n).astype(np.float32)
+        kept, cand = oracle.select_sampled(phi, B, R, noise)
+        r = min(R, B); m = n - r; E = n - B; C = min(2 * E, m)
+        assert len(kept) == B and np.all(np.diff(kept) > 0)
+        assert kept[B - r:].tolist() == list(range(m, n))                       # the recent pairs stay
+        evicted = np.setdiff1d(np.arange(m), kept)
+        assert len(evicted) == E and np.all(np.isin(evicted, cand))              # only candidates are evicted
+        # candidates are the C lowest scores (ties: the higher slot is the lower-ranked pair) - brute force
+        canon = np.where(np.isnan(phi[:m]), -np.inf, phi[:m]) + 0.0
+        order = sorted(range(m), key=lambda i: (canon[i], -i))
+        assert sorted(order[:C]) == cand.tolist()
+        # every non-candidate scores at least as high as every candidate
+        if C < m:
+            assert canon[np.setdiff1d(np.arange(m), cand)].min() >= canon[cand].max()
+
+
+def test_sampled_noise_decides_inside_the_candidate_set():
+    phi = np.array([0.9, 0.10, 0.8, 0.11, 0.12, 0.13, 0.7, 0.95], np.float32)    # n = 8, B = 6: E = 2, 4 candidates
+    kept, cand = oracle.select_sampled(phi, 6, 0, np.zeros(4, np.float32))
+    assert cand.tolist() == [1, 3, 4, 5] and kept.tolist() == [0, 2, 4, 5, 6, 7]
+    noise = np.array([-50.0, 0.0, 0.0, 50.0], np.float32)                         # rank 0 (slot 1) never, rank 3 (slot 5) surely
+    kept, _ = oracle.select_sampled(phi, 6, 0, noise)
+    assert 1 in kept and 5 not in kept and 3 not in kept                          # slot 3 is the lowest of the rest
+    # a pair outside the candidate set is never evicted, whatever the noise
+    for seed in range(50):
+        kept, _ = oracle.select_sampled(phi, 6, 0, np.random.default_rng(seed).gumbel(size=4).astype(np.float32) * 100)
+        assert all(s in kept for s in (0, 2, 6, 7))
+
+
+def test_sampled_matches_multinomial_without_replacement():
+    # The paper draws E pairs from Multinomial(softmax(-phi)) over the candidates.  Sequential draws
+    # without replacement have a closed form for every evicted SET (sum over the orders of
+    # p_a / 1 * p_b / (1 - p_a) ...); the Gumbel-perturbed selection must reproduce those
+    # probabilities.  A wrong sign of phi, a softmax over the wrong set, or drawing with replacement fails.
+    import itertools
+    phi = np.array([0.3, 2.0, -0.4, 0.9, 0.1, 1.5, 3.0], np.float32)   # n = 7, B = 5, R = 1: m = 6, E = 2, C = 4
+    B, R, E = 5, 1, 2
+    _, cand = oracle.select_sampled(phi, B, R, np.zeros(4, np.float32))
+    assert cand.tolist() == [0, 2, 3, 4]
+    logits = -phi[cand].astype(np.float64)
+    p = np.exp(logits - logits.max()); p /= p.sum()
+    exact = {}
+    for a, b in itertools.permutations(range(4), 2):
+        key = frozenset((int(cand[a]), int(cand[b])))
+        exact[key] = exact.get(key, 0.0) + p[a] * p[b] / (1.0 - p[a])
+    assert abs(sum(exact.values()) - 1.0) < 1e-12
+    rng = np.random.default_rng(7)
+    N = 40000
+    counts = {k: 0 for k in exact}
+    for _ in range(N):
+        kept, _c = oracle.select_sampled(phi, B, R, rng.gumbel(size=4).astype(np.float32))
+        ev = frozenset(int(x) for x in np.setdiff1d(np.arange(6), kept))
+        counts[ev] += 1
+    for k, pe in exact.items():
+        sigma = np.sqrt(pe * (1 - pe) / N)
+        assert abs(counts[k] / N - pe) < 5 * sigma + 1e-4, (sorted(k), counts[k] / N, pe)
