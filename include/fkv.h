@@ -141,6 +141,27 @@ int fkv_set_features(fkv_cache *c, int layer, int seq, const float *feat, void *
 int fkv_evict(fkv_cache *c, int layer, void *stream);
 
 /*
+ * evict(layer) with the paper's SAMPLED action - Section 3.1, second equation,
+ * and Appendix B.2: D = Multinomial_E(Softmax(Top_2E(-Phi))), s' = s \ D.  For
+ * every segment with n > B, E = n - B pairs are evicted: the candidates are
+ * the 2E competing pairs with the lowest scores (ties: the higher slot ranks
+ * lower; all competing pairs if there are fewer than 2E), and E of them are
+ * drawn without replacement with probabilities softmax(-score).  The draws use
+ * the CALLER'S randomness: noise holds standard Gumbel values g = -log(-log u),
+ * u uniform in (0, 1); the candidate of rank j in slot order uses g_j, and the
+ * E candidates with the largest (-score + g_j), compared in fp32, are evicted
+ * (Gumbel-top-k, which is sampling without replacement from the softmax; ties:
+ * the higher slot is evicted).  Everything else is as in fkv_evict.  With all
+ * g = 0 this is fkv_evict.
+ *
+ * noise: dev fp32 [layers of the call][max_batch][Hkv][noise_stride] (one
+ * layer, or all layers in order for FKV_ALL_LAYERS); noise_stride must be at
+ * least min(2E, n - R) for every segment that is evicted, else
+ * FKV_ERR_INVALID_ARG.  The library draws no random numbers itself.
+ */
+int fkv_evict_sampled(fkv_cache *c, int layer, const float *noise, int32_t noise_stride, void *stream);
+
+/*
  * decode_attn(q) - Appendix A: out[s][h] = sum_i softmax_i(scale <q[s][h], k_i>) v_i
  * over all retained pairs i of the KV head that query head h belongs to
  * (h / g).  q, out: dev [max_batch][Hkv*g][D] bf16.  scale 0 means 1/sqrt(D).
@@ -185,6 +206,9 @@ int fkv_score(fkv_cache *c, int layer, float *scores_out, void *stream);
  */
 int fkv_select(fkv_cache *c, int layer, const float *scores_in, int32_t *idx_out, int32_t *kept_count_out,
                void *stream);
+/* Selection by the sampled action of fkv_evict_sampled from given scores; noise dev [max_batch][Hkv][noise_stride]. */
+int fkv_select_sampled(fkv_cache *c, int layer, const float *scores_in, const float *noise, int32_t noise_stride,
+                       int32_t *idx_out, int32_t *kept_count_out, void *stream);
 /*
  * Compaction by given ascending slot lists (dev, layout as fkv_select writes
  * them; every (sequence) must have the same count on all its heads).

@@ -26,7 +26,7 @@ EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", 
            "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
            "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
            "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing",
-           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn"]
+           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled"]
 
 
 class FkvConfig(ctypes.Structure):
@@ -144,6 +144,11 @@ class Cache:
     def evict(self, layer=ALL_LAYERS):
         _check(lib().fkv_evict(self._h, layer, _stream()), "fkv_evict")
 
+    def evict_sampled(self, noise, layer=ALL_LAYERS):
+        """The paper's sampled action; noise [layers of the call][batch][Hkv][stride] standard Gumbel draws."""
+        _check(lib().fkv_evict_sampled(self._h, layer, _ptr(noise, torch.float32), int(noise.shape[-1]), _stream()),
+               "fkv_evict_sampled")
+
     def decode_attn(self, layer, q, out=None, scale=0.0):
         if out is None:
             out = torch.empty_like(q)
@@ -182,6 +187,14 @@ class Cache:
         cnt = torch.zeros((self.cfg.max_batch, self.cfg.num_kv_heads), dtype=torch.int32, device="cuda")
         _check(lib().fkv_select(self._h, layer, _ptr(scores, torch.float32), _ptr(idx, torch.int32),
                                 _ptr(cnt, torch.int32), _stream()), "fkv_select")
+        return idx, cnt
+
+    def select_sampled(self, layer, scores, noise):
+        idx = torch.full((self.cfg.max_batch, self.cfg.num_kv_heads, self.cap), -1, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros((self.cfg.max_batch, self.cfg.num_kv_heads), dtype=torch.int32, device="cuda")
+        _check(lib().fkv_select_sampled(self._h, layer, _ptr(scores, torch.float32), _ptr(noise, torch.float32),
+                                        int(noise.shape[-1]), _ptr(idx, torch.int32), _ptr(cnt, torch.int32), _stream()),
+               "fkv_select_sampled")
         return idx, cnt
 
     def compact(self, layer, idx, cnt):

@@ -160,6 +160,19 @@ int launch_score_any(fkv_cache *c, float *out, int seg_base, int tiles_bound, cu
                                 : launch_score<64>(c, out, seg_base, tiles_bound, st);
 }
 
+// One selection launch: mode 0 writes kept slot lists, mode 1 keep-priorities of the sampled action.
+void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float *scores, int32_t *idx,
+                   int32_t *kept_count, int seg_base, int fill_pages, float *prio, const float *noise, int noise_stride,
+                   int noise_base, cudaStream_t st) {
+  const bool single = max_old <= kSelRound;
+#define FKV_SEL(S, M) \
+  k_select<S, M><<<nblocks, kSelThreads, 0, st>>>(c->ctx, scores, idx, kept_count, seg_base, fill_pages, prio, noise, \
+                                                  noise_stride, noise_base)
+  if (mode == 0) { if (single) FKV_SEL(true, 0); else FKV_SEL(false, 0); }
+  else { if (single) FKV_SEL(true, 1); else FKV_SEL(false, 1); }
+#undef FKV_SEL
+}
+
 int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, int nwork_bound, cudaStream_t st) {
   dim3 grid((max_new + kCompactRows - 1) / kCompactRows, nwork_bound);
   if (grid.x == 0 || grid.y == 0) return FKV_OK;
@@ -414,7 +427,13 @@ int fkv_append(fkv_cache *c, int layer, const void *k, const void *v, const int3
   return FKV_OK;
 }
 
-int fkv_evict(fkv_cache *c, int layer, void *stream) {
+// Candidates the sampled action needs noise for in one segment: min(2E, competing pairs).
+static int sampled_candidates(int n, int B, int R) {
+  if (n <= B) return 0;
+  return std::min(2 * (n - B), n - std::min(R, B));
+}
+
+static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_stride, void *stream) {
   if (!c || (layer != FKV_ALL_LAYERS && !layer_ok(c, layer))) return FKV_ERR_INVALID_ARG;
   const int l0 = layer == FKV_ALL_LAYERS ? 0 : layer, l1 = layer == FKV_ALL_LAYERS ? c->cfg.num_layers : layer + 1;
   const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
@@ -426,6 +445,7 @@ int fkv_evict(fkv_cache *c, int layer, void *stream) {
       if (n > B) {
         for (int h = 0; h < Hkv; ++h)
           if (!c->loaded[(size_t)l * Hkv + h]) return FKV_ERR_NOT_READY;
+        if (noise && sampled_candidates(n, B, c->cfg.recent_keep) > noise_stride) return FKV_ERR_INVALID_ARG;
         nactive += Hkv;
         max_new = std::max(max_new, B);
         max_old = std::max(max_old, n);
@@ -442,8 +462,12 @@ int fkv_evict(fkv_cache *c, int layer, void *stream) {
   int rc = launch_score_any(c, c->ctx.scores, 0, (int)std::min<long long>(tiles, 1 << 30), st);
   if (rc) return rc;
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[2], st));
-  if (max_old <= kSelRound) k_select<true><<<nactive, kSelThreads, 0, st>>>(c->ctx, c->ctx.scores, c->ctx.idx, nullptr, 0, 1);
-  else k_select<false><<<nactive, kSelThreads, 0, st>>>(c->ctx, c->ctx.scores, c->ctx.idx, nullptr, 0, 1);
+  if (noise) {   // sampled action: scores -> keep-priorities (in place), then the same selection over them
+    launch_select(c, 1, max_old, nactive, c->ctx.scores, nullptr, nullptr, 0, 0, c->ctx.scores, noise, noise_stride,
+                  l0 * batch * Hkv, st);
+    FKV_LAUNCHED(c);
+  }
+  launch_select(c, 0, max_old, nactive, c->ctx.scores, c->ctx.idx, nullptr, 0, 1, nullptr, nullptr, 0, 0, st);
   FKV_LAUNCHED(c);
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[3], st));
   rc = launch_compact(c, c->ctx.idx, 0, max_new, nactive, st);
@@ -461,6 +485,13 @@ int fkv_evict(fkv_cache *c, int layer, void *stream) {
       n = std::min(n, c->h_budget[s]);
     }
   return FKV_OK;
+}
+
+int fkv_evict(fkv_cache *c, int layer, void *stream) { return evict_impl(c, layer, nullptr, 0, stream); }
+
+int fkv_evict_sampled(fkv_cache *c, int layer, const float *noise, int32_t noise_stride, void *stream) {
+  if (!noise || noise_stride < 1) return FKV_ERR_INVALID_ARG;
+  return evict_impl(c, layer, noise, noise_stride, stream);
 }
 
 int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream) {
@@ -519,22 +550,43 @@ int fkv_score(fkv_cache *c, int layer, float *scores_out, void *stream) {
   return launch_score_any(c, scores_out, layer * batch * Hkv, (int)tiles, st);
 }
 
-int fkv_select(fkv_cache *c, int layer, const float *scores_in, int32_t *idx_out, int32_t *kept_count_out,
-               void *stream) {
+static int select_impl(fkv_cache *c, int layer, const float *scores_in, const float *noise, int noise_stride,
+                       int32_t *idx_out, int32_t *kept_count_out, void *stream) {
   if (!c || !layer_ok(c, layer) || !scores_in || !idx_out || !kept_count_out) return FKV_ERR_INVALID_ARG;
   const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
+  if (noise)
+    for (int s = 0; s < batch; ++s)
+      if (sampled_candidates(c->h_len[(size_t)layer * batch + s], c->h_budget[s], c->cfg.recent_keep) > noise_stride)
+        return FKV_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   FKV_CUDA(cudaMemsetAsync(kept_count_out, 0, (size_t)batch * Hkv * 4, st));
   k_plan<<<1, 1024, 0, st>>>(c->ctx, layer, layer + 1, PLAN_SELECT, kScorePPS * kPage, nullptr);
   FKV_LAUNCHED(c);
   int max_old = 0;
   for (int s = 0; s < batch; ++s) max_old = std::max(max_old, c->h_len[(size_t)layer * batch + s]);
-  if (max_old <= kSelRound)
-    k_select<true><<<batch * Hkv, kSelThreads, 0, st>>>(c->ctx, scores_in, idx_out, kept_count_out, layer * batch * Hkv, 0);
-  else
-    k_select<false><<<batch * Hkv, kSelThreads, 0, st>>>(c->ctx, scores_in, idx_out, kept_count_out, layer * batch * Hkv, 0);
+  const float *sel_in = scores_in;
+  if (noise) {   // keep-priorities go to this layer's part of the workspace scratch
+    float *prio = c->ctx.scores + (size_t)layer * batch * Hkv * c->lay.cap;
+    launch_select(c, 1, max_old, batch * Hkv, scores_in, nullptr, nullptr, layer * batch * Hkv, 0, prio, noise,
+                  noise_stride, layer * batch * Hkv, st);
+    FKV_LAUNCHED(c);
+    sel_in = prio;
+  }
+  launch_select(c, 0, max_old, batch * Hkv, sel_in, idx_out, kept_count_out, layer * batch * Hkv, 0, nullptr, nullptr, 0,
+                0, st);
   FKV_LAUNCHED(c);
   return FKV_OK;
+}
+
+int fkv_select(fkv_cache *c, int layer, const float *scores_in, int32_t *idx_out, int32_t *kept_count_out,
+               void *stream) {
+  return select_impl(c, layer, scores_in, nullptr, 0, idx_out, kept_count_out, stream);
+}
+
+int fkv_select_sampled(fkv_cache *c, int layer, const float *scores_in, const float *noise, int32_t noise_stride,
+                       int32_t *idx_out, int32_t *kept_count_out, void *stream) {
+  if (!noise || noise_stride < 1) return FKV_ERR_INVALID_ARG;
+  return select_impl(c, layer, scores_in, noise, noise_stride, idx_out, kept_count_out, stream);
 }
 
 int fkv_compact(fkv_cache *c, int layer, const int32_t *idx, const int32_t *kept_count, void *stream) {

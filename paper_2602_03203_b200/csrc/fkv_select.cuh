@@ -52,12 +52,26 @@ __global__ void k_fill_pt_new(Ctx c, int seg0, int nseg) {
 // (so the bins follow the data, not fixed bit fields, and shared-memory
 // atomics spread out), picks the bin where the count from the top crosses k,
 // and narrows the window to it - at most three passes for 32-bit keys.
+//
+// MODE 1 is the first half of the sampled eviction action (Section 3.1, second equation; Appendix
+// B.2): the same search run for the m - 2E best pairs (E = pairs to evict) tells which 2E pairs
+// are the CANDIDATES (the lowest scores).  Instead of a slot list it writes a keep-priority per
+// slot: +infinity for a pair outside the candidate set, score - g_j for the candidate of rank j in
+// slot order, g_j the caller's standard Gumbel draw.  Keeping the best m - E priorities (a MODE 0
+// pass over them) then evicts exactly the E candidates with the largest -score + g: E draws
+// without replacement from softmax(-score) over the candidates.  prio may be the scores array.
 constexpr int kSelPerThread = 32;
 constexpr int kSelRound = kSelThreads * kSelPerThread;
 
-template <bool SINGLE>
+// Score back from its ordering key (canonical: -0 came in as +0, NaN as -infinity).
+__device__ __forceinline__ float key_score(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+template <bool SINGLE, int MODE>
 __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scores, int32_t *idx, int32_t *kept_count,
-                                                         int seg_base, int fill_pages) {
+                                                         int seg_base, int fill_pages, float *prio,
+                                                         const float *noise, int noise_stride, int noise_base) {
   __shared__ unsigned s_hist[kSelBins];
   __shared__ int s_scan[33];
   __shared__ unsigned s_red[64];
@@ -68,16 +82,30 @@ __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scor
   const SegPlan p = c.plan[seg];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (fill_pages) fill_pt_new(c, seg, p);
-  const int m = p.n_old - p.r, k = p.k_sel;
+  const int m = p.n_old - p.r;
+  const int k = MODE == 0 ? p.k_sel : max(0, m - 2 * (p.n_old - p.n_new));   // MODE 1: the non-candidates
   const float *sc = scores + (size_t)(seg - seg_base) * c.cap;
-  int32_t *out = idx + (size_t)(seg - seg_base) * c.cap;
-  if (kept_count && tid == 0) kept_count[seg - seg_base] = p.n_new;
-  // The protected recent slots close the list.
-  for (int j = tid; j < p.r; j += kSelThreads) out[k + j] = m + j;
-  if (k <= 0) return;
-  if (k >= m) {
-    for (int j = tid; j < m; j += kSelThreads) out[j] = j;
-    return;
+  int32_t *out = MODE == 0 ? idx + (size_t)(seg - seg_base) * c.cap : nullptr;
+  float *pr = MODE == 1 ? prio + (size_t)(seg - seg_base) * c.cap : nullptr;
+  const float *nz = MODE == 1 ? noise + (size_t)(seg - noise_base) * noise_stride : nullptr;
+  if (MODE == 0) {
+    if (kept_count && tid == 0) kept_count[seg - seg_base] = p.n_new;
+    // The protected recent slots close the list.
+    for (int j = tid; j < p.r; j += kSelThreads) out[k + j] = m + j;
+    if (k <= 0) return;
+    if (k >= m) {
+      for (int j = tid; j < m; j += kSelThreads) out[j] = j;
+      return;
+    }
+  } else {
+    if (k <= 0) {   // every competing pair is a candidate: rank = slot
+      for (int j = tid; j < m; j += kSelThreads) pr[j] = key_score(score_key(sc[j])) - nz[j];
+      return;
+    }
+    if (k >= m) {   // nothing to evict
+      for (int j = tid; j < m; j += kSelThreads) pr[j] = INFINITY;
+      return;
+    }
   }
   const int rounds = SINGLE ? 1 : (m + kSelRound - 1) / kSelRound;
   uint32_t key[kSelPerThread];
@@ -191,8 +219,14 @@ __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scor
 #pragma unroll
     for (int j = 0; j < kSelPerThread; ++j) {
       const bool g = j < nv && key[j] > T, e = j < nv && key[j] == T;
-      if (g) out[bgt + min(beq, need)] = slot0 + j;
-      else if (e && beq < need) out[bgt + beq] = slot0 + j;
+      if (MODE == 0) {
+        if (g) out[bgt + min(beq, need)] = slot0 + j;
+        else if (e && beq < need) out[bgt + beq] = slot0 + j;
+      } else if (j < nv) {
+        const bool kept = g || (e && beq < need);
+        const int rank = slot0 + j - (int)(bgt + min(beq, need));   // candidates before this slot
+        pr[slot0 + j] = kept ? INFINITY : key_score(key[j]) - nz[rank];
+      }
       bgt += g; beq += e;
     }
     run_gt += (unsigned)(tot & 0xffffffffu);

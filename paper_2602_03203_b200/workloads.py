@@ -23,7 +23,7 @@ from typing import List, Tuple
 import torch
 
 # Tensor ids that key the per-tensor random streams.
-_T_K, _T_V, _T_FEAT, _T_SCALE, _T_W, _T_Q, _T_NEW, _T_LEN, _T_SPIKE, _T_DUP = range(10)
+_T_K, _T_V, _T_FEAT, _T_SCALE, _T_W, _T_Q, _T_NEW, _T_LEN, _T_SPIKE, _T_DUP, _T_NOISE = range(11)
 
 FEATS_PER_HEAD = 6  # Appendix B.1: windows 8/16/32/L, cumulative sum, decayed sum
 CHUNK = 256         # Section 4.1: eviction length L = 256 (one "chunk" of queries)
@@ -200,6 +200,18 @@ def new_kv(w: Workload, layer: int, step: int = 0, device="cpu"):
     k = torch.randn((w.batch, w.num_kv_heads, w.head_dim), generator=g, device=device).to(torch.bfloat16)
     v = torch.randn((w.batch, w.num_kv_heads, w.head_dim), generator=g, device=device).to(torch.bfloat16)
     return k, v
+
+
+def gumbel_noise(w: Workload, layer: int, stride: int, event: int = 0, device="cpu") -> torch.Tensor:
+    """Standard Gumbel draws g = -log(-log u) for the sampled eviction action: [batch][Hkv][stride] fp32.
+
+    Random INPUT of the method (it has no arithmetic of the method in it): both the CPU oracle and the
+    CUDA path are handed the same values.
+    """
+    g = _gen(w, device, _T_NOISE, layer, 0, event)
+    u = torch.rand((w.batch, w.num_kv_heads, stride), generator=g, device=device, dtype=torch.float64)
+    u = u.clamp_(1e-12, 1.0 - 1e-12)
+    return (-torch.log(-torch.log(u))).to(torch.float32).contiguous()
 
 
 def segment_list(w: Workload) -> List[Tuple[int, int, int]]:

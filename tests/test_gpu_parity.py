@@ -445,3 +445,74 @@ def test_errors_are_status_codes():
         big.append(0, k.cuda(), v.cuda())
     assert e.value.code == -3                                        # capacity
     assert big.device_status()[0] == 0
+
+
+# ------------------------------------------------------------------ the sampled action (Section 3.1, Eq. 2; App. B.2)
+@pytest.mark.parametrize("n,B,R", [(512, 256, 0), (600, 344, 32), (5000, 4744, 0), (4097, 4096, 0), (9000, 8744, 256),
+                                   (300, 300, 0), (777, 100, 100), (1000, 600, 0), (40000, 39000, 0), (70001, 60000, 5)])
+@pytest.mark.parametrize("fn", [_normal, _ties, _special])
+def test_select_sampled_bit_exact(n, B, R, fn):
+    # Given the same scores and the same Gumbel draws the kept list is the oracle's, bit for bit
+    # (candidates, ranks, fp32 perturbation and ties all agree).
+    batch, Hkv = 2, 2
+    w = wl.Workload("sels", 1, Hkv, 4, 64, (n,) * batch, (B,) * batch, R, 13, "normal")
+    c = binding.from_workload(w)
+    for s in range(batch):
+        K, V, A, pos = wl.layer_inputs(w, 0, s, "cuda")
+        c.prefill(0, s, K, V, A, pos)
+    rng = np.random.default_rng(n * 7 + B + R)
+    sc = np.full((batch, Hkv, c.cap), np.nan, np.float32)
+    for s in range(batch):
+        for h in range(Hkv):
+            sc[s, h, :n] = fn(rng, n)
+    stride = max(1, min(2 * max(n - B, 0), n))
+    noise = wl.gumbel_noise(w, 0, stride)
+    if fn is _ties:
+        noise = torch.round(noise * 2) / 2        # ties among the perturbed values as well
+    idx, cnt = c.select_sampled(0, torch.from_numpy(sc).cuda(), noise.cuda())
+    idx, cnt = npf(idx), npf(cnt)
+    for s in range(batch):
+        for h in range(Hkv):
+            ref, _ = oracle.select_sampled(sc[s, h, :n], B, R, npf(noise)[s, h])
+            assert cnt[s, h] == len(ref)
+            assert np.array_equal(idx[s, h, :len(ref)], ref), (n, B, R, s, h)
+    assert c.device_status()[0] == 0
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 4])
+def test_evict_sampled_end_to_end(cfg):
+    w = small(cfg)
+    ld = Loaded(w)
+    stride = max(min(2 * (n - b), n) for n, b in zip(w.lens, w.budgets))
+    noise = torch.stack([wl.gumbel_noise(w, l, stride) for l in range(ld.L)])
+    gpu_scores = {l: npf(ld.cache.score(l)) for l in range(ld.L)}
+    ld.cache.evict_sampled(noise.cuda())
+    for l in range(ld.L):
+        for s in range(w.batch):
+            n, B = w.lens[s], w.budgets[s]
+            assert ld.cache.lengths(l)[s] == min(B, n)
+            for h in range(w.num_kv_heads):
+                K, V, A, pos = ld.head(l, s, h)
+                k2, v2, a2, p2 = ld.export(l, s, h)
+                kept_g = np.searchsorted(pos, p2).astype(np.int32)
+                ref, cand = oracle.select_sampled(gpu_scores[l][s, h, :n], B, w.recent_keep, npf(noise)[l, s, h])
+                assert np.array_equal(kept_g, ref)
+                assert np.array_equal(k2, K[kept_g]) and np.array_equal(v2, V[kept_g]) and np.array_equal(a2, A[kept_g])
+                assert np.all(np.diff(p2) > 0)
+    assert ld.cache.device_status()[0] == 0
+
+
+def test_evict_sampled_zero_noise_equals_evict_and_short_noise_is_rejected():
+    w = small(3)
+    a, b = Loaded(w), Loaded(w)
+    stride = 2 * (w.lens[0] - w.budgets[0])
+    a.cache.evict(binding.ALL_LAYERS)
+    b.cache.evict_sampled(torch.zeros((a.L, 1, w.num_kv_heads, stride), device="cuda"))
+    for l in range(a.L):
+        for h in range(w.num_kv_heads):
+            for x, y in zip(a.export(l, 0, h), b.export(l, 0, h)):
+                assert np.array_equal(x, y)
+    c = Loaded(w)
+    with pytest.raises(binding.FkvError) as e:
+        c.cache.evict_sampled(torch.zeros((a.L, 1, w.num_kv_heads, 8), device="cuda"))
+    assert e.value.code == -1
