@@ -93,6 +93,26 @@ def select_sampled(phi, B, R, noise):
     return kept[:nk].copy(), cand[:ncand.value].copy()
 
 
+def features(K, q, nvalid, A, scale=None, decay=0.9):
+    """Attention features refreshed at the end of a chunk (Appendix B.1).
+
+    K: [n][D] bf16 bits; q: [nq][g][D] bf16 bits (chronological); nvalid: [nq] pairs each query saw;
+    A: [n][6g] fp32 features before the chunk.  Returns the new [n][6g] array.
+    """
+    K, pK = _c(K, np.uint16)
+    q, pq = _c(q, np.uint16)
+    nvalid, pnv = _c(nvalid, np.int32)
+    A = np.array(A, dtype=np.float32, order="C", copy=True)
+    n, D = K.shape
+    nq, g, _ = q.shape
+    assert A.shape == (n, 6 * g) and nvalid.shape == (nq,)
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    lib().fkv_oracle_features(pK, n, D, g, pq, nq, pnv, ctypes.c_double(float(scale)), ctypes.c_double(float(decay)),
+                              A.ctypes.data_as(ctypes.c_void_p))
+    return A
+
+
 def compact(K, V, A, pos, kept):
     K, pK = _c(K, np.uint16)
     V, pV = _c(V, np.uint16)

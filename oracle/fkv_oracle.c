@@ -221,6 +221,55 @@ void fkv_oracle_attend(const uint16_t *q, const uint16_t *K, const uint16_t *V, 
 }
 
 /*
+ * Attention features of Appendix B.1 for one segment, refreshed at an eviction that closes a chunk
+ * of nq decode queries (chronological order, the last one the most recent).  Query t of query head j
+ * attended the first nvalid[t] pairs (the cache as it was then); its probabilities are
+ *   p_t = softmax(scale * <q_tj, k_i>) over i < nvalid[t],  0 for the pairs that did not exist yet.
+ * Per query head j the six features of pair i (reading of the paper's one-sentence description):
+ *   [0..2] recent windows 8, 16, 32:  (1/w) * sum of p_t[i] over the last min(w, nq) queries
+ *   [3]    window = the update length: (1/nq) * sum over all nq queries        (the chunk's score)
+ *   [4]    direct sum over chunks:     old[4] + chunk score
+ *   [5]    decayed sum:                decay * old[5] + chunk score            (decay 0.9 per chunk)
+ * A: [n][6g] in/out (a pair appended during the chunk comes in with zeros).  q: [nq][g][D] bf16.
+ */
+void fkv_oracle_features(const uint16_t *K, int n, int D, int g, const uint16_t *q, int nq, const int32_t *nvalid,
+                         double scale, double decay, float *A) {
+  static const int windows[3] = {8, 16, 32};
+  double *p = (double *)malloc((size_t)(n > 0 ? n : 1) * sizeof(double));
+  double *acc = (double *)calloc((size_t)(n > 0 ? n : 1) * 4, sizeof(double));
+  for (int j = 0; j < g; ++j) {
+    memset(acc, 0, (size_t)n * 4 * sizeof(double));
+    for (int t = 0; t < nq; ++t) {
+      int nv = nvalid[t] < n ? nvalid[t] : n;
+      double mx = -INFINITY, denom = 0.0;
+      for (int i = 0; i < nv; ++i) {
+        double dot = 0.0;
+        for (int c = 0; c < D; ++c)
+          dot += bf16_to_double(q[((size_t)t * g + j) * D + c]) * bf16_to_double(K[(size_t)i * D + c]);
+        p[i] = dot * scale;
+        if (p[i] > mx) mx = p[i];
+      }
+      for (int i = 0; i < nv; ++i) { p[i] = exp(p[i] - mx); denom += p[i]; }
+      int age = nq - 1 - t;   /* 0 = the most recent query */
+      for (int i = 0; i < nv; ++i) {
+        double pr = p[i] / denom;
+        for (int w = 0; w < 3; ++w) if (age < windows[w]) acc[(size_t)i * 4 + w] += pr;
+        acc[(size_t)i * 4 + 3] += pr;
+      }
+    }
+    for (int i = 0; i < n; ++i) {
+      float *a = A + (size_t)i * 6 * g + (size_t)j * 6;
+      double chunk = nq > 0 ? acc[(size_t)i * 4 + 3] / nq : 0.0;
+      for (int w = 0; w < 3; ++w) a[w] = (float)(acc[(size_t)i * 4 + w] / windows[w]);
+      a[3] = (float)chunk;
+      a[4] = (float)((double)a[4] + chunk);
+      a[5] = (float)(decay * (double)a[5] + chunk);
+    }
+  }
+  free(p); free(acc);
+}
+
+/*
  * One eviction step over many independent segments (score -> select ->
  * compact), the unit the CPU baseline times.  Segment i has n[i] pairs laid
  * out densely from offset off[i] (in pairs) in K, V, A, pos and phi; the

@@ -378,3 +378,70 @@ def test_sampled_matches_multinomial_without_replacement():
     for k, pe in exact.items():
         sigma = np.sqrt(pe * (1 - pe) / N)
         assert abs(counts[k] / N - pe) < 5 * sigma + 1e-4, (sorted(k), counts[k] / N, pe)
+
+
+# ---------------------------------------------------------------- attention features (Appendix B.1)
+def _rand_bits(rng, shape, scale=1.0):
+    return f32_to_bits((rng.standard_normal(shape) * scale).astype(np.float32))
+
+
+def test_features_uniform_attention_closed_form():
+    # Identical keys: every query spreads 1 / nvalid[t] over the pairs it saw, so every sum is known.
+    rng = np.random.default_rng(11)
+    n0, nq, g, D = 20, 40, 3, 16
+    K = np.repeat(_rand_bits(rng, (1, D)), n0 + nq, axis=0)
+    q = _rand_bits(rng, (nq, g, D))
+    nvalid = np.arange(n0 + 1, n0 + nq + 1, dtype=np.int32)          # one pair appended per query
+    A0 = np.zeros((n0 + nq, 6 * g), np.float32)
+    A0[:n0] = rng.random((n0, 6 * g)).astype(np.float32)
+    A1 = oracle.features(K, q, nvalid, A0)
+    for i in (0, 5, n0 - 1, n0, n0 + 7, n0 + nq - 1):
+        seen = [t for t in range(nq) if i < nvalid[t]]                # queries that could see pair i
+        for j in range(g):
+            row = A1[i, 6 * j:6 * j + 6]
+            for k, w in enumerate((8, 16, 32)):
+                expect = sum(1.0 / nvalid[t] for t in seen if nq - 1 - t < w) / w
+                assert abs(row[k] - expect) < 1e-6
+            chunk = sum(1.0 / nvalid[t] for t in seen) / nq
+            assert abs(row[3] - chunk) < 1e-6
+            assert abs(row[4] - (A0[i, 6 * j + 4] + chunk)) < 1e-6
+            assert abs(row[5] - (0.9 * A0[i, 6 * j + 5] + chunk)) < 1e-6
+    # a pair appended at the last step was seen by one query only: window-8 feature = (1/n)/8
+    assert abs(A1[n0 + nq - 1, 0] - 1.0 / (n0 + nq) / 8) < 1e-7
+
+
+def test_features_against_library_softmax_and_one_hot():
+    rng = np.random.default_rng(12)
+    n, nq, g, D = 50, 24, 2, 32
+    Kb, qb = _rand_bits(rng, (n, D)), _rand_bits(rng, (nq, g, D))
+    nvalid = np.full(nq, n, np.int32)
+    A1 = oracle.features(Kb, qb, nvalid, np.zeros((n, 6 * g), np.float32), scale=0.3)
+    Kf = torch.from_numpy(bits_to_f64(Kb)); qf = torch.from_numpy(bits_to_f64(qb))
+    P = torch.softmax(torch.einsum("tjd,nd->jtn", qf, Kf) * 0.3, dim=-1).numpy()     # [g][nq][n], library softmax
+    for j in range(g):
+        assert np.allclose(A1[:, 6 * j + 0], P[j, -8:].sum(0) / 8, atol=1e-6)
+        assert np.allclose(A1[:, 6 * j + 1], P[j, -16:].sum(0) / 16, atol=1e-6)
+        assert np.allclose(A1[:, 6 * j + 2], P[j].sum(0) / 32, atol=1e-6)             # only 24 queries, still / 32
+        assert np.allclose(A1[:, 6 * j + 3], P[j].mean(0), atol=1e-6)
+    # a query far along one key puts all its mass there
+    Kone = np.zeros((4, D), np.float32); Kone[2, 0] = 50.0
+    qone = np.zeros((1, 1, D), np.float32); qone[0, 0, 0] = 50.0
+    A2 = oracle.features(f32_to_bits(Kone), f32_to_bits(qone), np.array([4], np.int32), np.zeros((4, 6), np.float32),
+                         scale=1.0)
+    assert np.allclose(A2[2], [1 / 8, 1 / 16, 1 / 32, 1.0, 1.0, 1.0]) and np.allclose(A2[[0, 1, 3]], 0.0)
+
+
+def test_features_chunks_accumulate_and_decay():
+    rng = np.random.default_rng(13)
+    n, g, D = 30, 2, 16
+    Kb = _rand_bits(rng, (n, D))
+    nv = np.full(10, n, np.int32)
+    q1, q2 = _rand_bits(rng, (10, g, D)), _rand_bits(rng, (10, g, D))
+    Z = np.zeros((n, 6 * g), np.float32)
+    A1 = oracle.features(Kb, q1, nv, Z)
+    A2 = oracle.features(Kb, q2, nv, A1)
+    c1, c2 = oracle.features(Kb, q1, nv, Z)[:, 3::6], oracle.features(Kb, q2, nv, Z)[:, 3::6]
+    assert np.allclose(A2[:, 4::6], c1 + c2, atol=1e-6)                 # direct sum over chunks
+    assert np.allclose(A2[:, 5::6], 0.9 * c1 + c2, atol=1e-6)           # per-chunk decay 0.9
+    assert np.allclose(A2[:, 3::6], c2, atol=1e-7)                      # window features belong to the last chunk only
+    assert np.allclose(A2[:, 3::6].sum(0), 1.0, atol=1e-5)              # mean of probability rows still sums to 1
