@@ -78,6 +78,9 @@ typedef struct {
   int32_t max_tokens_per_head; /* capacity of one segment, n <= this */
   int32_t num_pages;           /* pages in the pool; 0 = enough for every segment at capacity
                                   plus the transient copies of an all-layer eviction */
+  int32_t feature_window;      /* W: decode queries kept on record per (layer, sequence) for the attention
+                                  features of Appendix B.1 (a multiple of 8, <= 512; the paper's update
+                                  length L, e.g. 256); 0 = the library does not maintain the features */
 } fkv_config;
 
 /* Bytes of device workspace fkv_init_cache needs for this config. */
@@ -215,6 +218,25 @@ int fkv_select_sampled(fkv_cache *c, int layer, const float *scores_in, const fl
  * Syncs (reads the new lengths back).
  */
 int fkv_compact(fkv_cache *c, int layer, const int32_t *idx, const int32_t *kept_count, void *stream);
+
+/*
+ * Attention features a_n of Appendix B.1, maintained by the library when feature_window > 0.
+ * Every fkv_append_decode_attn / fkv_decode_step records the token's queries, their softmax
+ * statistics and the number of pairs they saw (the last W tokens since the last eviction).
+ * fkv_evict / fkv_evict_sampled then refresh the features of the segments they evict, before
+ * scoring: per query head, in this order inside a_n,
+ *   windows 8, 16, 32: (1/w) sum over the last w recorded queries of the softmax probability
+ *                      the head gave the pair (0 for queries older than the pair),
+ *   window = chunk:    the same mean over all recorded queries of the chunk (the chunk's score),
+ *   direct sum:        previous value + chunk score,
+ *   decayed sum:       0.9 * previous value + chunk score,
+ * and start a new chunk.  With no query on record (e.g. right after fkv_prefill) the stored
+ * features are used as they are.  The paper gives one sentence on these features; mean versus sum,
+ * and what a chunk is, are this library's reading of it.
+ * fkv_update_features does the refresh alone for `layer` (all its sequences), without closing the
+ * chunk - a staged entry point for checks.  FKV_ERR_NOT_READY if feature_window is 0.
+ */
+int fkv_update_features(fkv_cache *c, int layer, void *stream);
 
 /* Row stride, in elements, of the score and index arrays above. */
 int fkv_score_stride(const fkv_cache *c, int32_t *cap);

@@ -26,13 +26,13 @@ EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", 
            "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
            "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
            "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing",
-           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled"]
+           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled", "fkv_update_features"]
 
 
 class FkvConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "num_layers", "num_kv_heads", "group_size", "head_dim", "max_batch", "page_size", "scorer_hidden",
-        "activation", "budget", "recent_keep", "max_tokens_per_head", "num_pages")]
+        "activation", "budget", "recent_keep", "max_tokens_per_head", "num_pages", "feature_window")]
 
 
 class FkvError(RuntimeError):
@@ -79,11 +79,11 @@ class Cache:
     """One budgeted KV cache on the current CUDA device (see include/fkv.h for the semantics)."""
 
     def __init__(self, num_layers, num_kv_heads, group_size, head_dim, max_batch, budget, max_tokens_per_head,
-                 recent_keep=0, activation=ACT_RELU, num_pages=0, page_size=16, scorer_hidden=16):
+                 recent_keep=0, activation=ACT_RELU, num_pages=0, page_size=16, scorer_hidden=16, feature_window=0):
         if not torch.cuda.is_available():
             raise RuntimeError("fkv needs a CUDA device; there is no CPU path")
         self.cfg = FkvConfig(num_layers, num_kv_heads, group_size, head_dim, max_batch, page_size, scorer_hidden,
-                             activation, budget, recent_keep, max_tokens_per_head, num_pages)
+                             activation, budget, recent_keep, max_tokens_per_head, num_pages, feature_window)
         nbytes = ctypes.c_size_t(0)
         _check(lib().fkv_workspace_bytes(ctypes.byref(self.cfg), ctypes.byref(nbytes)), "fkv_workspace_bytes")
         self.workspace_bytes = nbytes.value
@@ -197,6 +197,9 @@ class Cache:
                "fkv_select_sampled")
         return idx, cnt
 
+    def update_features(self, layer):
+        _check(lib().fkv_update_features(self._h, layer, _stream()), "fkv_update_features")
+
     def compact(self, layer, idx, cnt):
         _check(lib().fkv_compact(self._h, layer, _ptr(idx, torch.int32), _ptr(cnt, torch.int32), _stream()),
                "fkv_compact")
@@ -284,18 +287,18 @@ def workspace_bytes_for(w, num_layers=None, num_pages=0, max_tokens=None) -> int
     """Bytes of device workspace ``from_workload`` would allocate (no device access)."""
     cfg = FkvConfig(num_layers or w.num_layers, w.num_kv_heads, w.group_size, w.head_dim, w.batch, w.page_size,
                     w.scorer_hidden, w.activation, max(w.budgets), w.recent_keep,
-                    max_tokens or (max(w.lens) + 256), num_pages)
+                    max_tokens or (max(w.lens) + 256), num_pages, 0)
     nbytes = ctypes.c_size_t(0)
     _check(lib().fkv_workspace_bytes(ctypes.byref(cfg), ctypes.byref(nbytes)), "fkv_workspace_bytes")
     return nbytes.value
 
 
-def from_workload(w, num_layers=None, num_pages=0, max_tokens=None) -> Cache:
+def from_workload(w, num_layers=None, num_pages=0, max_tokens=None, feature_window=0) -> Cache:
     """A cache shaped for a ``workloads.Workload`` with per-sequence budgets set."""
     L = num_layers or w.num_layers
     c = Cache(L, w.num_kv_heads, w.group_size, w.head_dim, w.batch, max(w.budgets),
               max_tokens or (max(w.lens) + 256), recent_keep=w.recent_keep, activation=w.activation,
-              num_pages=num_pages)
+              num_pages=num_pages, feature_window=feature_window)
     for s, b in enumerate(w.budgets):
         if b != max(w.budgets):
             c.set_budget(s, b)

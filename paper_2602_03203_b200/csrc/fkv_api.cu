@@ -17,6 +17,7 @@
 #include "fkv_aux.cuh"
 #include "fkv_compact.cuh"
 #include "fkv_dev.cuh"
+#include "fkv_features.cuh"
 #include "fkv_score.cuh"
 #include "fkv_select.cuh"
 
@@ -33,7 +34,7 @@ constexpr size_t kMaxSmem = 227 * 1024;
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, total;
+  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, hist_q, hist_ml, hist_n, hist_cnt, total;
   int cap, max_pages, num_pages, page_bytes, F, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
 };
 
@@ -47,6 +48,7 @@ bool valid_config(const fkv_config *c) {
   if (c->activation < 0 || c->activation > 3) return false;
   if (c->budget < 1 || c->recent_keep < 0 || c->max_tokens_per_head < 1 || c->num_pages < 0) return false;
   if ((int64_t)c->num_layers * c->max_batch * c->num_kv_heads > (1 << 20)) return false;
+  if (c->feature_window < 0 || c->feature_window > 512 || c->feature_window % 8) return false;
   return true;
 }
 
@@ -83,6 +85,11 @@ Layout make_layout(const fkv_config &c) {
   L.work = take(nseg * 4);
   L.tile1 = take((nseg + 1) * 4);
   L.seq_tickets = take((size_t)c.num_layers * c.max_batch * 4);
+  const size_t ls = (size_t)c.num_layers * c.max_batch, W = (size_t)c.feature_window, Hq = (size_t)c.num_kv_heads * c.group_size;
+  L.hist_q = take(ls * W * Hq * D * 2);
+  L.hist_ml = take(ls * W * Hq * 8);
+  L.hist_n = take(ls * W * 4);
+  L.hist_cnt = take(W ? ls * 4 : 0);
   L.total = off;
   return L;
 }
@@ -107,6 +114,7 @@ struct fkv_cache {
   std::vector<uint8_t> staging;
   uint64_t launches = 0;
   int sm_count = 148;
+  float feature_scale = 0.f;  // softmax scale of the recorded queries (the last decode call's)
   int max_cluster = 0;  // largest attention cluster this device places (found at the first launch)
   bool timing = false, timed = false;
   cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -171,6 +179,29 @@ void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float
   if (mode == 0) { if (single) FKV_SEL(true, 0); else FKV_SEL(false, 0); }
   else { if (single) FKV_SEL(true, 1); else FKV_SEL(false, 1); }
 #undef FKV_SEL
+}
+
+// Attention features of the segments on the work list (after a k_plan): grid (page groups, work items).
+constexpr int kFeatWarps = 8;
+template <int D>
+int launch_features_t(fkv_cache *c, int max_old, int nwork_bound, float scale_log2, cudaStream_t st) {
+  const size_t smem = FeatSmem::bytes(D, kFeatWarps, c->cfg.feature_window);
+  static bool attr_done = false;
+  if (!attr_done) {
+    FKV_CUDA(cudaFuncSetAttribute(k_features<D, kFeatWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)FeatSmem::bytes(D, kFeatWarps, 512)));
+    attr_done = true;
+  }
+  dim3 grid(((max_old + kPage - 1) / kPage + kFeatWarps - 1) / kFeatWarps, nwork_bound);
+  if (grid.x == 0 || grid.y == 0) return FKV_OK;
+  k_features<D, kFeatWarps><<<grid, kFeatWarps * 32, smem, st>>>(c->ctx, scale_log2);
+  FKV_LAUNCHED(c);
+  return FKV_OK;
+}
+int launch_features(fkv_cache *c, int max_old, int nwork_bound, cudaStream_t st) {
+  const float scale_log2 = c->feature_scale * 1.4426950408889634f;
+  return c->cfg.head_dim == 128 ? launch_features_t<128>(c, max_old, nwork_bound, scale_log2, st)
+                                : launch_features_t<64>(c, max_old, nwork_bound, scale_log2, st);
 }
 
 int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, int nwork_bound, cudaStream_t st) {
@@ -247,6 +278,7 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
     splits *= 2;
   const int pps = std::max(1, (maxpages + splits - 1) / splits);
   if (scale == 0.f) scale = 1.f / sqrtf((float)D);
+  if (app) c->feature_scale = scale;
   AttendArgs a;
   a.layer = layer; a.q = (const __nv_bfloat16 *)q; a.out = (__nv_bfloat16 *)out;
   a.scale_log2 = scale * 1.4426950408889634f; a.pps = pps; a.append = app ? 1 : 0;
@@ -292,6 +324,8 @@ int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, voi
   x.scores = (float *)(ws + L.scores); x.idx = (int *)(ws + L.idx); x.plan = (SegPlan *)(ws + L.plan);
   x.work = (int *)(ws + L.work); x.tile1_start = (int *)(ws + L.tile1);
   x.seq_tickets = (int *)(ws + L.seq_tickets);
+  x.hist_w = cfg->feature_window; x.hist_q = ws + L.hist_q; x.hist_ml = (float *)(ws + L.hist_ml);
+  x.hist_n = (int *)(ws + L.hist_n); x.hist_cnt = (int *)(ws + L.hist_cnt);
   c->h_len.assign((size_t)cfg->num_layers * cfg->max_batch, 0);
   c->h_budget.assign(cfg->max_batch, cfg->budget);
   c->loaded.assign((size_t)cfg->num_layers * cfg->num_kv_heads, 0);
@@ -458,6 +492,10 @@ static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_str
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[0], st));
   k_plan<<<1, 1024, 0, st>>>(c->ctx, l0, l1, PLAN_EVICT, kScorePPS * kPage, nullptr);
   FKV_LAUNCHED(c);
+  if (c->cfg.feature_window > 0 && c->feature_scale > 0.f) {   // refresh a_n from the chunk's recorded queries first
+    const int rcf = launch_features(c, max_old, nactive, st);
+    if (rcf) return rcf;
+  }
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[1], st));
   int rc = launch_score_any(c, c->ctx.scores, 0, (int)std::min<long long>(tiles, 1 << 30), st);
   if (rc) return rc;
@@ -527,6 +565,20 @@ int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *p
     if (rc) return rc;
   }
   return FKV_OK;
+}
+
+int fkv_update_features(fkv_cache *c, int layer, void *stream) {
+  if (!c || !layer_ok(c, layer)) return FKV_ERR_INVALID_ARG;
+  if (c->cfg.feature_window == 0) return FKV_ERR_NOT_READY;
+  if (c->feature_scale == 0.f) return FKV_OK;   // no query has been recorded yet
+  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
+  int max_old = 0;
+  for (int s = 0; s < batch; ++s) max_old = std::max(max_old, c->h_len[(size_t)layer * batch + s]);
+  if (max_old == 0) return FKV_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  k_plan<<<1, 1024, 0, st>>>(c->ctx, layer, layer + 1, PLAN_SCORE_ALL, kScorePPS * kPage, nullptr);
+  FKV_LAUNCHED(c);
+  return launch_features(c, max_old, batch * Hkv, st);
 }
 
 int fkv_score_stride(const fkv_cache *c, int32_t *cap) {

@@ -63,7 +63,7 @@ struct AttendArgs {
   __nv_bfloat16 *out;       // same
   float scale_log2;         // softmax scale times log2(e)
   int pps;                  // pages per split (>= 1); ceil(pages / pps) <= gridDim.x for every segment
-  int append;               // 1: append k_new / v_new at slot n first
+  int append;               // 1: append k_new / v_new at slot n first (and record the query when the cache keeps a history)
   const uint8_t *k_new, *v_new;  // [batch][Hkv][D] bf16
   const int32_t *pos_new;   // [batch] or null (last position + 1)
   unsigned long long seq_mask;   // sequences that append (0 = all)
@@ -113,6 +113,11 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
   const bool tail = app && active && pg1 == npages;     // this CTA's range holds the new pair
   const bool fresh = tail && (n_old % kPage) == 0;      // ... which opens a new page: nothing to copy for it
   const size_t qrow0 = ((size_t)seq * c.Hkv + head) * G;  // first query head of the group
+  // Query record for the attention features: ring slot of this token in the (layer, sequence) history.
+  const bool rec = app && c.hist_w > 0;
+  const int hcnt = rec ? c.hist_cnt[a.layer * c.batch + seq] : 0;
+  const size_t hrow = ((size_t)(a.layer * c.batch + seq) * (rec ? c.hist_w : 1) + (rec ? hcnt % c.hist_w : 0)) * (c.Hkv * G) +
+                      (size_t)head * G;   // first query head of the group in the record
 
   const size_t ring_bytes = AttendSmem::ring(D, NCW, SLOTS);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + ring_bytes);                      // full[SLOTS], empty[SLOTS]
@@ -338,7 +343,11 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
       acc = fmaf(f, recv_o[s * per + e], acc);
     }
     a.out[qrow0 * D + ge] = __float2bfloat16(L > 0.f ? acc / L : 0.f);   // an empty sequence gives zeros
+    if (rec && ge - r * D == 0) reinterpret_cast<float2 *>(c.hist_ml)[hrow + r] = make_float2(M, L);
   }
+  if (rec && rank == 0)   // the queries themselves: G rows of D bf16
+    for (int i = tid; i < G * D / 8; i += blockDim.x)
+      reinterpret_cast<uint4 *>(c.hist_q + hrow * D * 2)[i] = reinterpret_cast<const uint4 *>(a.q + qrow0 * D)[i];
 
   // ---- the length grows once every CTA of the sequence (all heads, all splits) has read the old one ----
   if (app && tid == 0) {
@@ -348,6 +357,10 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
     if (tk == total - 1) {
       *ticket = 0;
       c.len[a.layer * c.batch + seq] = n_old + 1;
+      if (rec) {
+        c.hist_n[(size_t)(a.layer * c.batch + seq) * c.hist_w + hcnt % c.hist_w] = n_old + 1;
+        c.hist_cnt[a.layer * c.batch + seq] = hcnt + 1;
+      }
     }
   }
 }

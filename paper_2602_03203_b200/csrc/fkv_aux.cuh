@@ -13,6 +13,8 @@ __global__ void k_reset(Ctx c) {
   for (int i = t0; i < c.num_pages; i += stride) c.free_stack[i] = c.num_pages - 1 - i;
   for (int i = t0; i < c.L * c.batch; i += stride) c.len[i] = 0;
   for (int i = t0; i < c.L * c.batch; i += stride) c.seq_tickets[i] = 0;
+  if (c.hist_w)
+    for (int i = t0; i < c.L * c.batch; i += stride) c.hist_cnt[i] = 0;
   if (t0 == 0) {
     c.ctrl[CTRL_FREE_TOP] = c.num_pages;
     c.ctrl[CTRL_STATUS] = 0;
@@ -220,7 +222,10 @@ __global__ void k_commit(Ctx c, int l0, int l1) {
     c.free_stack[push + i] = ptrow[i];
     if (i < cnt_new) ptrow[i] = ptnew[i];
   }
-  if (threadIdx.x == 0 && seg % c.Hkv == 0) c.len[seg / c.Hkv] = p.n_new;
+  if (threadIdx.x == 0 && seg % c.Hkv == 0) {
+    c.len[seg / c.Hkv] = p.n_new;
+    if (c.hist_w) c.hist_cnt[seg / c.Hkv] = 0;   // the eviction closed the chunk: its query record starts over
+  }
 }
 
 }  // namespace fkv

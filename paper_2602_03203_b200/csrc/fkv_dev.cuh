@@ -62,6 +62,12 @@ struct Ctx {
   int *tile1_start;  // prefix of score tiles over the work list
   int *planhdr;
   int *seq_tickets;  // [L][batch]
+  // Record of the decode queries of the current chunk (attention-feature maintenance; hist_w = 0: off).
+  int hist_w;          // ring capacity W in queries
+  uint8_t *hist_q;     // [L][batch][W][Hkv * G][D] bf16
+  float *hist_ml;      // [L][batch][W][Hkv * G][2]: softmax max and sum of that query (log2 domain)
+  int *hist_n;         // [L][batch][W]: pairs the query saw
+  int *hist_cnt;       // [L][batch]: queries recorded since the last eviction
 };
 
 __device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head) {

@@ -1,0 +1,118 @@
+"""Attention-feature maintenance (Appendix B.1) against the oracle: the library records the decode
+queries of a chunk and recomputes every pair's window and cumulative features at the eviction."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from harness import kept_set_within_band
+from paper_2602_03203_b200 import binding, workloads as wl
+from util import bits, npf
+
+pytestmark = pytest.mark.gpu
+
+FEAT_ATOL, FEAT_RTOL = 2e-6, 2e-3     # probabilities <= 1; bf16 products accumulated in fp32 vs fp64
+SCORE_TOL = 1e-3
+
+
+def _run_chunk(w, W, steps, L=None):
+    """Prefill, then `steps` fused append+attention tokens; returns the cache and the host-side history."""
+    L = L or w.num_layers
+    c = binding.from_workload(w, L, feature_window=W)
+    st = {}
+    for l in range(L):
+        c.load_scorers(l, *wl.scorer_params(w, l))
+        for s in range(w.batch):
+            K, V, A, pos = wl.layer_inputs(w, l, s)
+            c.prefill(l, s, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
+            for h in range(w.num_kv_heads):
+                st[(l, s, h)] = dict(K=bits(K)[h], V=bits(V)[h], A=npf(A)[h].copy(), q=[], nv=[])
+    g = w.group_size
+    for step in range(steps):
+        for l in range(L):
+            k, v = wl.new_kv(w, l, step)
+            q = wl.queries(w, l, step)
+            c.append_decode_attn(l, k.cuda(), v.cuda(), q.cuda())
+            kb, vb, qb = bits(k), bits(v), bits(q)
+            for s in range(w.batch):
+                for h in range(w.num_kv_heads):
+                    d = st[(l, s, h)]
+                    d["K"] = np.concatenate([d["K"], kb[s, h][None]]); d["V"] = np.concatenate([d["V"], vb[s, h][None]])
+                    d["A"] = np.concatenate([d["A"], np.zeros((1, d["A"].shape[1]), np.float32)])
+                    d["q"].append(qb[s, h * g:(h + 1) * g]); d["nv"].append(len(d["K"]))
+    return c, st
+
+
+def _expected(d, W):
+    q = np.stack(d["q"][-W:]); nv = np.array(d["nv"][-W:], np.int32)     # the ring keeps the last W queries
+    return oracle.features(d["K"], q, nv, d["A"])
+
+
+@pytest.mark.parametrize("g,D,W,steps", [(4, 128, 64, 40), (4, 128, 32, 45), (7, 128, 40, 40), (4, 64, 64, 33),
+                                         (1, 128, 16, 7), (8, 64, 24, 50)])
+def test_update_features_matches_oracle(g, D, W, steps):
+    w = wl.Workload("feat", 2, 2, g, D, (100, 37), (1 << 20,) * 2, 0, 51, "normal")
+    c, st = _run_chunk(w, W, steps)
+    for l in range(2):
+        c.update_features(l)
+    for (l, s, h), d in st.items():
+        _, _, a2, _ = c.export_head(l, s, h)
+        exp = _expected(d, W)
+        got = npf(a2)
+        assert got.shape == exp.shape
+        assert np.all(np.abs(got - exp) <= FEAT_ATOL + FEAT_RTOL * np.abs(exp)), (l, s, h, np.abs(got - exp).max())
+    assert c.device_status()[0] == 0
+
+
+def test_no_recorded_query_leaves_features_alone():
+    w = wl.Workload("feat0", 1, 2, 4, 128, (200,), (100,), 0, 52, "normal")
+    c, st = _run_chunk(w, 32, 0)
+    c.update_features(0)
+    c.evict(0)                       # one-shot compression after prefill: the prefilled features are scored
+    for h in range(2):
+        d = st[(0, 0, h)]
+        W1, b1, W2, b2 = (npf(t)[h] for t in wl.scorer_params(w, 0))
+        phi = oracle.score(d["K"], d["V"], d["A"], W1, b1, W2, float(b2))
+        kept = oracle.select(phi, 100, 0)
+        _, _, a2, p2 = c.export_head(0, 0, h)
+        assert kept_set_within_band(phi, kept, npf(p2), 200, 100, 0, SCORE_TOL)
+        assert np.array_equal(npf(a2), d["A"][npf(p2)])
+
+
+def test_decode_evict_cycle_with_maintained_features():
+    # Two chunks of L tokens with an eviction after each (the protocol of Section 3.1, R = L): the scorer
+    # sees features the library derived from its own record; the oracle is fed the same queries.
+    B, Lev = 128, 32
+    w = wl.Workload("featcyc", 1, 2, 4, 128, (B,), (B,), Lev, 53, "channel_lognormal")
+    c = binding.from_workload(w, feature_window=Lev)
+    c.load_scorers(0, *wl.scorer_params(w, 0))
+    K, V, A, pos = wl.layer_inputs(w, 0, 0)
+    c.prefill(0, 0, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
+    st = {h: dict(K=bits(K)[h], V=bits(V)[h], A=npf(A)[h].copy(), pos=npf(pos).copy()) for h in range(2)}
+    g = w.group_size
+    W1, b1, W2, b2 = (npf(t) for t in wl.scorer_params(w, 0))
+    for chunk in range(2):
+        qs = {h: [] for h in range(2)}; nvs = {h: [] for h in range(2)}
+        for step in range(Lev):
+            k, v = wl.new_kv(w, 0, chunk * Lev + step); q = wl.queries(w, 0, chunk * Lev + step)
+            c.append_decode_attn(0, k.cuda(), v.cuda(), q.cuda())
+            for h in range(2):
+                d = st[h]
+                d["K"] = np.concatenate([d["K"], bits(k)[0, h][None]]); d["V"] = np.concatenate([d["V"], bits(v)[0, h][None]])
+                d["A"] = np.concatenate([d["A"], np.zeros((1, 6 * g), np.float32)])
+                d["pos"] = np.concatenate([d["pos"], [d["pos"][-1] + 1]]).astype(np.int32)
+                qs[h].append(bits(q)[0, h * g:(h + 1) * g]); nvs[h].append(len(d["K"]))
+        c.evict(0)
+        assert c.lengths(0) == [B]
+        for h in range(2):
+            d = st[h]
+            A1 = oracle.features(d["K"], np.stack(qs[h]), np.array(nvs[h], np.int32), d["A"])
+            phi = oracle.score(d["K"], d["V"], A1, W1[h], b1[h], W2[h], float(b2[h]))
+            kept = oracle.select(phi, B, Lev)
+            _, _, a2, p2 = c.export_head(0, 0, h)
+            kept_g = np.searchsorted(d["pos"], npf(p2)).astype(np.int32)
+            assert kept_set_within_band(phi, kept, kept_g, len(phi), B, Lev, SCORE_TOL)
+            got = npf(a2)
+            assert np.all(np.abs(got - A1[kept_g]) <= FEAT_ATOL + FEAT_RTOL * np.abs(A1[kept_g]))
+            st[h] = dict(K=d["K"][kept_g], V=d["V"][kept_g], A=got.copy(), pos=d["pos"][kept_g])   # follow the GPU's state
+    assert c.device_status()[0] == 0
