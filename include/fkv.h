@@ -79,8 +79,9 @@ typedef struct {
   int32_t num_pages;           /* pages in the pool; 0 = enough for every segment at capacity
                                   plus the transient copies of an all-layer eviction */
   int32_t feature_window;      /* W: decode queries kept on record per (layer, sequence) for the attention
-                                  features of Appendix B.1 (a multiple of 8, <= 512; the paper's update
-                                  length L, e.g. 256); 0 = the library does not maintain the features */
+                                  features of Appendix B.1 (a multiple of 8, at most 328 for D = 128;
+                                  the paper's update length L, e.g. 256); 0 = the library does not
+                                  maintain the features */
 } fkv_config;
 
 /* Bytes of device workspace fkv_init_cache needs for this config. */
@@ -259,12 +260,12 @@ int fkv_sync_lengths(fkv_cache *c, void *stream);
 
 /*
  * Per-kernel timing of fkv_evict.  While on, fkv_evict records CUDA events on
- * the caller's stream around its five kernels; fkv_get_evict_timing waits for
- * the last recorded set and returns milliseconds for
- * {plan, score, select, compact, commit}.
+ * the caller's stream around its kernels; fkv_get_evict_timing waits for the
+ * last recorded set and returns milliseconds for
+ * {plan, score, select (both passes of the sampled action), compact, commit, feature refresh}.
  */
 int fkv_set_timing(fkv_cache *c, int on);
-int fkv_get_evict_timing(fkv_cache *c, float ms_out[5]);
+int fkv_get_evict_timing(fkv_cache *c, float ms_out[6]);
 
 /* Number of kernel launches this handle has enqueued so far. */
 int fkv_launch_count(const fkv_cache *c, uint64_t *launches);

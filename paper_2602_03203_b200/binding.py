@@ -245,10 +245,10 @@ class Cache:
         _check(lib().fkv_set_timing(self._h, int(on)), "fkv_set_timing")
 
     def evict_timing(self):
-        """Milliseconds of the last timed fkv_evict: dict plan/score/select/compact/commit."""
-        arr = (ctypes.c_float * 5)()
+        """Milliseconds of the last timed fkv_evict: dict plan/score/select/compact/commit/features."""
+        arr = (ctypes.c_float * 6)()
         _check(lib().fkv_get_evict_timing(self._h, arr), "fkv_get_evict_timing")
-        return dict(zip(("plan", "score", "select", "compact", "commit"), (float(x) for x in arr)))
+        return dict(zip(("plan", "score", "select", "compact", "commit", "features"), (float(x) for x in arr)))
 
     def launch_count(self):
         n = ctypes.c_uint64(0)

@@ -30,6 +30,7 @@ thread_local std::string g_cuda_error;
 constexpr int kScorePPS = 8;  // consumer warps of the scorer = pages per tile
 constexpr int kAttendMinPages = 4;
 constexpr size_t kMaxSmem = 227 * 1024;
+constexpr int kFeatWarps = 8;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -48,7 +49,8 @@ bool valid_config(const fkv_config *c) {
   if (c->activation < 0 || c->activation > 3) return false;
   if (c->budget < 1 || c->recent_keep < 0 || c->max_tokens_per_head < 1 || c->num_pages < 0) return false;
   if ((int64_t)c->num_layers * c->max_batch * c->num_kv_heads > (1 << 20)) return false;
-  if (c->feature_window < 0 || c->feature_window > 512 || c->feature_window % 8) return false;
+  if (c->feature_window < 0 || c->feature_window % 8) return false;
+  if (c->feature_window && FeatSmem::bytes(c->head_dim, kFeatWarps, c->feature_window) > kMaxSmem) return false;
   return true;
 }
 
@@ -117,7 +119,7 @@ struct fkv_cache {
   float feature_scale = 0.f;  // softmax scale of the recorded queries (the last decode call's)
   int max_cluster = 0;  // largest attention cluster this device places (found at the first launch)
   bool timing = false, timed = false;
-  cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t ev[7] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};  // [6]: after the plan
 };
 
 namespace {
@@ -182,17 +184,16 @@ void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float
 }
 
 // Attention features of the segments on the work list (after a k_plan): grid (page groups, work items).
-constexpr int kFeatWarps = 8;
 template <int D>
 int launch_features_t(fkv_cache *c, int max_old, int nwork_bound, float scale_log2, cudaStream_t st) {
   const size_t smem = FeatSmem::bytes(D, kFeatWarps, c->cfg.feature_window);
-  static bool attr_done = false;
-  if (!attr_done) {
-    FKV_CUDA(cudaFuncSetAttribute(k_features<D, kFeatWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)FeatSmem::bytes(D, kFeatWarps, 512)));
-    attr_done = true;
+  static size_t attr_bytes = 0;   // largest opt-in made so far
+  if (smem > attr_bytes) {
+    FKV_CUDA(cudaFuncSetAttribute(k_features<D, kFeatWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_bytes = smem;
   }
-  dim3 grid(((max_old + kPage - 1) / kPage + kFeatWarps - 1) / kFeatWarps, nwork_bound);
+  const int group = kFeatWarps * kFeatPPW;   // pages per CTA
+  dim3 grid(((max_old + kPage - 1) / kPage + group - 1) / group, nwork_bound);
   if (grid.x == 0 || grid.y == 0) return FKV_OK;
   k_features<D, kFeatWarps><<<grid, kFeatWarps * 32, smem, st>>>(c->ctx, scale_log2);
   FKV_LAUNCHED(c);
@@ -492,6 +493,7 @@ static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_str
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[0], st));
   k_plan<<<1, 1024, 0, st>>>(c->ctx, l0, l1, PLAN_EVICT, kScorePPS * kPage, nullptr);
   FKV_LAUNCHED(c);
+  if (tm) FKV_CUDA(cudaEventRecord(c->ev[6], st));
   if (c->cfg.feature_window > 0 && c->feature_scale > 0.f) {   // refresh a_n from the chunk's recorded queries first
     const int rcf = launch_features(c, max_old, nactive, st);
     if (rcf) return rcf;
@@ -713,11 +715,13 @@ int fkv_set_timing(fkv_cache *c, int on) {
   return FKV_OK;
 }
 
-int fkv_get_evict_timing(fkv_cache *c, float ms_out[5]) {
+int fkv_get_evict_timing(fkv_cache *c, float ms_out[6]) {
   if (!c || !ms_out) return FKV_ERR_INVALID_ARG;
   if (!c->timed) return FKV_ERR_NOT_READY;
   FKV_CUDA(cudaEventSynchronize(c->ev[5]));
   for (int i = 0; i < 5; ++i) FKV_CUDA(cudaEventElapsedTime(&ms_out[i], c->ev[i], c->ev[i + 1]));
+  FKV_CUDA(cudaEventElapsedTime(&ms_out[5], c->ev[6], c->ev[1]));   // feature refresh: after the plan, before the scorer
+  ms_out[0] -= ms_out[5];
   return FKV_OK;
 }
 

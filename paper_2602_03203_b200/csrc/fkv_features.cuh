@@ -16,8 +16,10 @@
 // pays 2 g D + 12 g bytes per token for the record instead of a read-modify-write of every pair's
 // feature row per token.
 //
-// grid (groups of NW pages, work list); NW warps, warp w owns page w of the group: its K fragments
-// stay in registers while the CTA walks the query heads, staging one head's queries at a time.
+// grid (groups of NW * PPW pages, work list); NW warps, each owning PPW pages of the group.  Only the K
+// rows of the pages are staged (16-byte async copies keep the record's swizzle); the CTA walks the
+// query heads with two query buffers: the next head's queries stream in (async copies again) while
+// the current head is computed.
 #pragma once
 #include "fkv_dev.cuh"
 
@@ -25,23 +27,39 @@ namespace fkv {
 
 constexpr float kFeatDecay = 0.9f;   // Appendix B.1: per-chunk decay of the decayed sum
 
+constexpr int kFeatPPW = 1;   // pages per warp
+
 struct FeatSmem {
-  // pages [nw][4D * 16] | queries of one head [W][2D] | M [W] | 1/L [W] | pairs seen [W]
+  // K rows of the pages [nw * PPW][16][2D] | their meta rows [nw * PPW][16 * 49 words, padded] |
+  // 2 x { queries of one head [W][2D] | M + log2 L [W] | pairs seen [W] }
+  static constexpr size_t kMeta = 16 * 49 * 4 + 64;   // room for the widest meta block (g = 8), 16-byte multiple
+  static __host__ __device__ size_t qbuf(int D, int W) { return (size_t)W * 2 * D + (size_t)W * 8; }
   static __host__ __device__ size_t bytes(int D, int nw, int W) {
-    return (size_t)nw * 4 * D * kPage + (size_t)W * 2 * D + (size_t)W * 12 + 16;
+    return (size_t)nw * kFeatPPW * (2 * D * kPage + kMeta) + 2 * qbuf(D, W) + 16;
   }
 };
 
+// 2^x for x <= 0 (tiny results may flush to zero).
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Offset of 16-byte chunk ch of row r in a [rows][2D bytes] tile whose chunks are XOR-swizzled by the row index.
+__device__ __forceinline__ int row_chunk_off(int r, int ch, int D) {
+  return r * 2 * D + ((ch >> 3) << 7) + (((ch & 7) ^ (r & 7)) << 4);
+}
+
 template <int D, int NW>
 __global__ void __launch_bounds__(NW * 32) k_features(Ctx c, float scale_log2) {
-  constexpr int KSH = D / 16;
-  constexpr int PAGE_KV = 4 * D * kPage;
+  constexpr int KSH = D / 16, NCH = D / 8, PPW = kFeatPPW, PG = NW * PPW;
+  constexpr int PAGE_K = 2 * D * kPage;
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ uint64_t s_bar;
   if ((int)blockIdx.y >= c.planhdr[PH_NWORK]) return;
   const int seg = c.work[blockIdx.y];
   const int n = c.plan[seg].n_old;
-  const int npages = (n + kPage - 1) / kPage, pg0 = blockIdx.x * NW;
+  const int npages = (n + kPage - 1) / kPage, pg0 = blockIdx.x * PG;
   if (pg0 >= npages) return;
   const int ls = seg / c.Hkv, head = seg % c.Hkv, G = c.G, W = c.hist_w, Hq = c.Hkv * G;
   const int cnt = c.hist_cnt[ls];
@@ -50,118 +68,155 @@ __global__ void __launch_bounds__(NW * 32) k_features(Ctx c, float scale_log2) {
   const int Lp = (Lc + 7) & ~7;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
   const int gid = lane >> 2, tig = lane & 3;
-  uint8_t *pages = smem;
-  uint8_t *qs = smem + (size_t)NW * PAGE_KV;                       // [Lp][2D], 16-byte chunks swizzled by row
-  float *sM = reinterpret_cast<float *>(qs + (size_t)W * 2 * D), *sIL = sM + W;
-  int *sN = reinterpret_cast<int *>(sIL + W);
-  const int np = min(NW, npages - pg0);
+  uint8_t *kpages = smem;
+  uint8_t *metas = smem + (size_t)PG * PAGE_K;                     // the pages' meta blocks (features + positions)
+  uint8_t *qbuf0 = metas + (size_t)PG * FeatSmem::kMeta;           // two buffers of FeatSmem::qbuf bytes
+  const size_t qbytes = FeatSmem::qbuf(D, W);
+  const int np = min(PG, npages - pg0);
 
-  // ---- the K|V blocks of this group's pages: one bulk copy each, one barrier ----
-  if (tid == 0) {
-    mbar_init(smem_u32(&s_bar), 1);
-    fence_barrier_init();
+  // ---- K rows of this group's pages: 16-byte async copies, chunk for chunk (the swizzle is kept) ----
+  for (int e = tid; e < np * kPage * NCH; e += blockDim.x) {
+    const int pg = e / (kPage * NCH), rc = e - pg * (kPage * NCH), r = rc / NCH, ch = rc - r * NCH;
+    const int pid = c.pt[(size_t)seg * c.max_pages + pg0 + pg];
+    cp_async16(smem_u32(kpages + (size_t)pg * PAGE_K + r * 2 * D + ch * 16),
+               c.pool + (size_t)pid * c.page_bytes + (size_t)r * 4 * D + ch * 16);
   }
-  __syncthreads();
-  if (warp == 0) {
-    if (lane == 0) mbar_arrive_expect_tx(smem_u32(&s_bar), (uint32_t)(np * PAGE_KV));
-    __syncwarp();
-    if (lane < np) {
-      const int pid = c.pt[(size_t)seg * c.max_pages + pg0 + lane];
-      bulk_g2s(smem_u32(pages + (size_t)lane * PAGE_KV), c.pool + (size_t)pid * c.page_bytes, PAGE_KV, smem_u32(&s_bar));
-    }
+  const int meta_chunks = (kPage * (c.F + 1) * 4) / 16;   // the meta block is a multiple of 16 bytes (64 (F + 1))
+  for (int e = tid; e < np * meta_chunks; e += blockDim.x) {
+    const int pg = e / meta_chunks, ch = e - pg * meta_chunks;
+    const int pid = c.pt[(size_t)seg * c.max_pages + pg0 + pg];
+    cp_async16(smem_u32(metas + (size_t)pg * FeatSmem::kMeta + ch * 16), c.pool + (size_t)pid * c.page_bytes + c.off_f + ch * 16);
   }
-  const bool ok = mbar_wait(smem_u32(&s_bar), 0);
-  if (!ok) set_status(c, kDevWaitTimeout);   // falls through: every thread still reaches the barriers below
-
-  // K rows of this warp's page as A fragments (keys x channels), for all heads.
-  uint32_t ka[KSH][4];
-  const int krow = ((lane >> 3) & 1) * 8 + (lane & 7), khi = lane >> 4;
-  if (warp < np) {
-    const uint32_t kbase = smem_u32(pages + (size_t)warp * PAGE_KV);
-#pragma unroll
-    for (int ks = 0; ks < KSH; ++ks) ldsm_x4(ka[ks], kbase + kv_chunk_off(krow, ks * 2 + khi, D));
-  }
-  const int slot0 = (pg0 + warp) * kPage + gid;   // this lane's pairs: slot0 and slot0 + 8
   const uint8_t *hq = c.hist_q + (size_t)ls * W * Hq * D * 2;
   const float2 *hml = reinterpret_cast<const float2 *>(c.hist_ml) + (size_t)ls * W * Hq;
   const int *hn = c.hist_n + (size_t)ls * W;
-  // ldmatrix roles for the queries as B (queries x channels, row-major): matrix mi -> 8 queries,
-  // channel chunk 2 * kp * 2 + mi: one x4 load gives the B fragments of two k-steps.
+  const int newest = (cnt - 1) % W;                  // ring slot of the most recent query (cnt >= 1 here)
+  const int nv_min = hn[(cnt - Lc) % W];             // the oldest recorded query saw the fewest pairs
+  // ldmatrix roles.  K as A (keys x channels): matrix lane/8 -> keys ((lane/8)&1)*8.., chunk +lane/16.
+  // Queries as B (queries x channels, row-major): matrix lane/8 -> chunk +lane/8; one x4 = two k-steps.
+  const int krow = ((lane >> 3) & 1) * 8 + (lane & 7), khi = lane >> 4;
   const int qrow = lane & 7, qmi = lane >> 3;
 
-  for (int j = 0; j < G; ++j) {
+  // Stages head j's queries newest first (index a = age) into buffer b: the vectors by async copies, the
+  // statistics through registers.  Rows beyond the record are zero / "saw nothing".
+  auto stage = [&](int j, int b) {
     const int qh = head * G + j;
-    __syncthreads();   // the previous head's queries are no longer read
-    // ---- stage this head's queries newest first (index a = age), with their statistics ----
-    for (int e = tid; e < Lp * (D / 8); e += blockDim.x) {
-      const int a = e / (D / 8), ch = e - a * (D / 8);
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    uint8_t *qs = qbuf0 + (size_t)b * qbytes;
+    float *sM = reinterpret_cast<float *>(qs + (size_t)W * 2 * D);
+    int *sN = reinterpret_cast<int *>(sM + W);
+    for (int e = tid; e < Lp * NCH; e += blockDim.x) {
+      const int a = e / NCH, ch = e - a * NCH;
+      uint8_t *dst = qs + row_chunk_off(a, ch, D);
       if (a < Lc) {
-        const int hs = ((cnt - 1 - a) % W + W) % W;
-        v = *reinterpret_cast<const uint4 *>(hq + ((size_t)hs * Hq + qh) * D * 2 + ch * 16);
+        const int hs = newest - a + (newest < a ? W : 0);
+        cp_async16(smem_u32(dst), hq + ((size_t)hs * Hq + qh) * D * 2 + ch * 16);
+      } else {
+        *reinterpret_cast<uint4 *>(dst) = make_uint4(0u, 0u, 0u, 0u);
       }
-      *reinterpret_cast<uint4 *>(qs + (size_t)a * 2 * D + ((ch & ~7) | ((ch ^ a) & 7)) * 16) = v;
     }
     for (int a = tid; a < Lp; a += blockDim.x) {
-      float M = 0.f, il = 0.f;
+      float Mp = 0.f;
       int nv = 0;
       if (a < Lc) {
-        const int hs = ((cnt - 1 - a) % W + W) % W;
+        const int hs = newest - a + (newest < a ? W : 0);
         const float2 ml = hml[(size_t)hs * Hq + qh];
-        M = ml.x; il = 1.f / ml.y; nv = hn[hs];
+        Mp = ml.x + log2f(ml.y); nv = hn[hs];
       }
-      sM[a] = M; sIL[a] = il; sN[a] = nv;
+      sM[a] = Mp; sN[a] = nv;
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  stage(0, 0);   // (its group also carries the page copies issued above)
+
+  for (int j = 0; j < G; ++j) {
+    const uint8_t *qs = qbuf0 + (size_t)(j & 1) * qbytes;
+    const float *sM = reinterpret_cast<const float *>(qs + (size_t)W * 2 * D);
+    const int *sN = reinterpret_cast<const int *>(sM + W);
+    __syncthreads();   // the other buffer (head j - 1) is no longer read
+    if (j + 1 < G) {
+      stage(j + 1, (j + 1) & 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");   // head j (and the pages) have landed; j + 1 is in flight
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
-    if (warp >= np) continue;
-    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // rows gid, gid + 8: windows 8, 16, 32, all
     const uint32_t qbase = smem_u32(qs);
-    for (int a0 = 0; a0 < Lp; a0 += 8) {
-      float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+    for (int u = 0; u < PPW; ++u) {
+      const int pg = warp * PPW + u;
+      if (pg >= np) break;
+      // K rows of the page as A fragments.
+      uint32_t ka[KSH][4];
+      const uint32_t kbase = smem_u32(kpages + (size_t)pg * PAGE_K);
 #pragma unroll
-      for (int kp = 0; kp < KSH / 2; ++kp) {
-        uint32_t b[4];
-        const int r = a0 + qrow, ch = kp * 4 + qmi;
-        ldsm_x4(b, qbase + r * 2 * D + (((ch & ~7) | ((ch ^ r) & 7)) << 4));
-        mma_bf16(s, ka[2 * kp][0], ka[2 * kp][1], ka[2 * kp][2], ka[2 * kp][3], b[0], b[1]);
-        mma_bf16(s, ka[2 * kp + 1][0], ka[2 * kp + 1][1], ka[2 * kp + 1][2], ka[2 * kp + 1][3], b[2], b[3]);
+      for (int ks = 0; ks < KSH; ++ks) ldsm_x4(ka[ks], kbase + row_chunk_off(krow, ks * 2 + khi, D));
+      const int slot0 = (pg0 + pg) * kPage + gid;   // this lane's pairs: slot0 and slot0 + 8
+      const bool whole = (pg0 + pg) * kPage + kPage <= nv_min;   // every recorded query saw the whole page
+      float run0 = 0.f, run1 = 0.f;                 // running sums over the queries, newest first
+      float w8[2] = {0.f, 0.f}, w16[2] = {0.f, 0.f}, w32[2] = {0.f, 0.f};
+      for (int a0 = 0; a0 < Lp; a0 += 8) {
+        if (a0 == 8) { w8[0] = run0; w8[1] = run1; }
+        if (a0 == 16) { w16[0] = run0; w16[1] = run1; }
+        if (a0 == 32) { w32[0] = run0; w32[1] = run1; }
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int kp = 0; kp < KSH / 2; ++kp) {
+          uint32_t b[4];
+          ldsm_x4(b, qbase + row_chunk_off(a0 + qrow, kp * 4 + qmi, D));
+          mma_bf16(sa, ka[2 * kp][0], ka[2 * kp][1], ka[2 * kp][2], ka[2 * kp][3], b[0], b[1]);
+          mma_bf16(sb, ka[2 * kp + 1][0], ka[2 * kp + 1][1], ka[2 * kp + 1][2], ka[2 * kp + 1][3], b[2], b[3]);
+        }
+        // [0], [1]: pair slot0, queries a0 + 2 tig (+1); [2], [3]: pair slot0 + 8.
+        const float2 M2 = *reinterpret_cast<const float2 *>(sM + a0 + 2 * tig);
+        float p00 = ex2((sa[0] + sb[0]) * scale_log2 - M2.x), p01 = ex2((sa[1] + sb[1]) * scale_log2 - M2.y);
+        float p10 = ex2((sa[2] + sb[2]) * scale_log2 - M2.x), p11 = ex2((sa[3] + sb[3]) * scale_log2 - M2.y);
+        if (!whole) {
+          const int2 N2 = *reinterpret_cast<const int2 *>(sN + a0 + 2 * tig);
+          if (slot0 >= N2.x) p00 = 0.f;
+          if (slot0 >= N2.y) p01 = 0.f;
+          if (slot0 + 8 >= N2.x) p10 = 0.f;
+          if (slot0 + 8 >= N2.y) p11 = 0.f;
+        } else if (a0 + 8 > Lc) {   // the padded tail of the query axis
+          if (a0 + 2 * tig >= Lc) { p00 = 0.f; p10 = 0.f; }
+          if (a0 + 2 * tig + 1 >= Lc) { p01 = 0.f; p11 = 0.f; }
+        }
+        run0 += p00 + p01;
+        run1 += p10 + p11;
       }
-      // s[0], s[1]: pair slot0, queries a0 + 2 tig (+1); s[2], s[3]: pair slot0 + 8.
+      if (Lp <= 8) { w8[0] = run0; w8[1] = run1; }
+      if (Lp <= 16) { w16[0] = run0; w16[1] = run1; }
+      if (Lp <= 32) { w32[0] = run0; w32[1] = run1; }
+      float vals[2][4] = {{w8[0], w16[0], w32[0], run0}, {w8[1], w16[1], w32[1], run1}};
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int a = a0 + 2 * tig + e;
-        const float M = sM[a], il = sIL[a];
-        const int nv = sN[a];
-        const float p0 = slot0 < nv ? exp2f(s[e] * scale_log2 - M) * il : 0.f;
-        const float p1 = slot0 + 8 < nv ? exp2f(s[2 + e] * scale_log2 - M) * il : 0.f;
-        if (a0 < 8) { acc[0][0] += p0; acc[1][0] += p1; }
-        if (a0 < 16) { acc[0][1] += p0; acc[1][1] += p1; }
-        if (a0 < 32) { acc[0][2] += p0; acc[1][2] += p1; }
-        acc[0][3] += p0; acc[1][3] += p1;
+      for (int r = 0; r < 2; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          vals[r][k] += __shfl_xor_sync(0xffffffffu, vals[r][k], 1);
+          vals[r][k] += __shfl_xor_sync(0xffffffffu, vals[r][k], 2);
+        }
+      // Lane tig == r of a quad writes row r's six features of this head (rows gid and gid + 8).
+      if (tig < 2) {
+        const int slot = slot0 + 8 * tig;
+        if (slot < n) {
+          const float a8 = tig ? vals[1][0] : vals[0][0], a16 = tig ? vals[1][1] : vals[0][1];
+          const float a32 = tig ? vals[1][2] : vals[0][2], all = tig ? vals[1][3] : vals[0][3];
+          float *f = reinterpret_cast<float *>(metas + (size_t)pg * FeatSmem::kMeta) + (slot % kPage) * (c.F + 1) + j * 6;
+          const float chunk = all / (float)Lc;
+          f[0] = a8 * (1.f / 8.f); f[1] = a16 * (1.f / 16.f); f[2] = a32 * (1.f / 32.f);
+          f[3] = chunk;
+          f[4] = f[4] + chunk;
+          f[5] = fmaf(kFeatDecay, f[5], chunk);
+        }
       }
     }
-#pragma unroll
-    for (int r = 0; r < 2; ++r)
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        acc[r][k] += __shfl_xor_sync(0xffffffffu, acc[r][k], 1);
-        acc[r][k] += __shfl_xor_sync(0xffffffffu, acc[r][k], 2);
-      }
-    // Lane tig == r of a quad writes row r's six features of this head (rows gid and gid + 8).
-    if (tig < 2) {
-      const int slot = slot0 + 8 * tig;
-      if (slot < n) {
-        const float w8 = tig ? acc[1][0] : acc[0][0], w16 = tig ? acc[1][1] : acc[0][1];
-        const float w32 = tig ? acc[1][2] : acc[0][2], wall = tig ? acc[1][3] : acc[0][3];
-        const int pid = c.pt[(size_t)seg * c.max_pages + slot / kPage];
-        float *f = meta_row(c, c.pool + (size_t)pid * c.page_bytes, slot % kPage) + j * 6;
-        const float chunk = wall / (float)Lc;
-        f[0] = w8 * (1.f / 8.f); f[1] = w16 * (1.f / 16.f); f[2] = w32 * (1.f / 32.f);
-        f[3] = chunk;
-        f[4] = f[4] + chunk;
-        f[5] = fmaf(kFeatDecay, f[5], chunk);
-      }
-    }
+  }
+  // ---- the refreshed meta blocks go back to their page records (every row was written by one lane) ----
+  __syncthreads();
+  for (int e = tid; e < np * meta_chunks; e += blockDim.x) {
+    const int pg = e / meta_chunks, ch = e - pg * meta_chunks;
+    const int pid = c.pt[(size_t)seg * c.max_pages + pg0 + pg];
+    *reinterpret_cast<uint4 *>(c.pool + (size_t)pid * c.page_bytes + c.off_f + ch * 16) =
+        *reinterpret_cast<const uint4 *>(metas + (size_t)pg * FeatSmem::kMeta + ch * 16);
   }
 }
 
