@@ -284,6 +284,14 @@ def run_ours(args):
     dom = "score" if kern["score"] >= kern["compact"] else "compact"
     dom_bytes = eb[dom]
     achieved = dom_bytes / (kern[dom] * 1e-3) / 1e9
+    # DRAM traffic of the dominant kernel from its ncu capture on a 4-layer slice of this workload
+    # (profiles/k_score_cfg3_4layers.md, profiles/k_compact_cfg3_4layers.md), scaled by the units of the launch:
+    # 616.2 B per scored pair; 1174 B (read + write) per kept pair at B = 8192 only.
+    traffic = args.traffic
+    if traffic is None and args.config == 3:
+        pairs = L * w.num_kv_heads * sum(n for n, b in zip(w.lens, w.budgets) if n > b)
+        kept = L * w.num_kv_heads * sum(b for n, b in zip(w.lens, w.budgets) if n > b)
+        traffic = 616.2 * pairs if dom == "score" else (1174.0 * kept if max(w.budgets) == 8192 else None)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": N, "steps": args.steps, "warmup": args.warmup,
@@ -304,7 +312,7 @@ def run_ours(args):
         "decode_note": "attention side only (append + GQA attention, one launch per layer, layers of a token "
                        "overlap); no projections, MLP or sampling",
         "roofline": {"bound": "hbm", "kernel": f"k_{dom}", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": args.traffic},
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic},
         "e2e": {"value": N * eb["total"] / (e_evict * 1e-3) / 1e9, "unit": UNIT,
                 "decode_tokens_per_s": N * w.batch * T / (e_decode * 1e-3) if T else 0.0,
                 "h2d_bytes_per_step": kh.numel() * 2 + vh.numel() * 2 + qh.numel() * 2,
