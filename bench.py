@@ -17,6 +17,7 @@ dominant kernel and the CPU oracle's timing ride along.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -197,7 +198,14 @@ def run_ours(args):
     w = wl.config(args.config, budget=args.budget)
     L = args.layers or w.num_layers
     T = args.decode_tokens
-    cache = binding.from_workload(w, L, max_tokens=max(w.lens) + max(256, T))
+    # Config 2 is the decode protocol of Section 3.1: the cache sits at the budget, grows by L = recent_keep
+    # tokens, and is evicted back.  Its step is one such chunk: T decode tokens FIRST, then the eviction
+    # (with --feature-window the tokens' queries are recorded and the eviction refreshes the features first).
+    chunk_mode = args.config == 2
+    if chunk_mode:
+        T = args.decode_tokens = w.recent_keep if args.decode_tokens == 16 else args.decode_tokens
+        w = dataclasses.replace(w, lens=tuple(min(n, b) for n, b in zip(w.lens, w.budgets)))
+    cache = binding.from_workload(w, L, max_tokens=max(w.lens) + max(256, T), feature_window=args.feature_window)
     for l in range(L):
         cache.load_scorers(l, *wl.scorer_params(w, l, dev))
         for s in range(w.batch):
@@ -220,7 +228,8 @@ def run_ours(args):
     kept_dev = torch.empty((L, w.batch, w.num_kv_heads, max(w.budgets)), dtype=torch.int32, device=dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)        # > 126 MB of L2
 
-    eb = evict_bytes(w, L)
+    w_ev = dataclasses.replace(w, lens=tuple(n + T for n in w.lens)) if chunk_mode else w   # lengths at the eviction
+    eb = evict_bytes(w_ev, L)
     lens_after = [min(n, b) for n, b in zip(w.lens, w.budgets)]
     dec_bytes = sum(decode_bytes_per_token(w, L, [n + t + 1 for n in lens_after]) for t in range(T))
     cache.set_timing(True)
@@ -234,6 +243,17 @@ def run_ours(args):
         if e2e:
             kd.copy_(kh, non_blocking=True); vd.copy_(vh, non_blocking=True); qd.copy_(qh, non_blocking=True)
         ev[1].record()
+        if chunk_mode:
+            for t in range(T):
+                cache.decode_step(kd[t], vd[t], qd[t], od[t])
+            ev[2].record()
+            cache.evict(binding.ALL_LAYERS)
+            if e2e:
+                oh.copy_(od, non_blocking=True)
+            ev[3].record()
+            torch.cuda.synchronize()
+            return dict(h2d=ev[0].elapsed_time(ev[1]), decode=ev[1].elapsed_time(ev[2]), evict=ev[2].elapsed_time(ev[3]),
+                        kernels=cache.evict_timing())
         cache.evict(binding.ALL_LAYERS)
         ev[2].record()
         for t in range(T):
@@ -260,11 +280,14 @@ def run_ours(args):
     e2e_res = [one_step(True) for _ in range(max(1, min(args.steps, 3)))]
     # The paper's sampled action (Top-2E candidates, E Gumbel-top-k draws) on the same workload: one
     # more selection pass per eviction.  Reported beside the deterministic step, not instead of it.
-    stride = max(min(2 * (n - b), n) for n, b in zip(w.lens, w.budgets) if n > b)
+    stride = max(min(2 * (n - b), n) for n, b in zip(w_ev.lens, w_ev.budgets) if n > b)
     noise = torch.stack([wl.gumbel_noise(w, l, stride, device=dev) for l in range(L)])
     sampled_ms = []
     for _ in range(4):
         cache.restore(snap); flush.fill_(1); torch.cuda.synchronize()
+        if chunk_mode:
+            for t in range(T):
+                cache.decode_step(kd[t], vd[t], qd[t], od[t])
         ev[0].record(); cache.evict_sampled(noise); ev[1].record(); torch.cuda.synchronize()
         sampled_ms.append(ev[0].elapsed_time(ev[1]))
     sampled_ms = ranks.max(min(sampled_ms[1:]))
@@ -298,8 +321,11 @@ def run_ours(args):
         "ms_per_step": evict_ms + decode_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "layers": L, "kv_heads": w.num_kv_heads, "group_size": w.group_size,
-                   "head_dim": w.head_dim, "batch": w.batch, "context": max(w.lens), "budget": max(w.budgets),
+                   "head_dim": w.head_dim, "batch": w.batch, "context": max(w_ev.lens), "budget": max(w.budgets),
                    "recent_keep": w.recent_keep, "decode_tokens_per_step": T, "parallelism": f"replicas{N}",
+                   "step": "T decode tokens, then one all-layer eviction" if chunk_mode else
+                           "one all-layer eviction, then T decode tokens",
+                   "feature_window": args.feature_window,
                    "l2": "cache restored and a 512 MiB buffer overwritten before every step; inputs exceed L2"},
         "evict_ms": evict_ms, "decode_ms": decode_ms, "kernel_ms": kern,
         "evict_bytes": eb, "evict_frac_of_measured_peak": value / N / peak,
@@ -321,7 +347,7 @@ def run_ours(args):
         "gpu_launches": launches, "clocks": clocks,
     }
     if ranks.rank == 0 and N == 1 and not args.no_cpu_baseline:
-        smp = oracle_sample(w)
+        smp = oracle_sample(w_ev)
         line["cpu_baseline"] = {
             "value": smp["bytes"] / smp["seconds"] / 1e9, "unit": UNIT, "cores": smp["threads"], "kind": "oracle",
             "sample": f"{smp['layers']} of {w.num_layers} layers ({smp['pairs']} pairs), score+select+compact, "
@@ -341,6 +367,8 @@ def main():
     ap.add_argument("--budget", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None, help="fewer layers (profiling captures only)")
     ap.add_argument("--decode-tokens", type=int, default=16)
+    ap.add_argument("--feature-window", type=int, default=0,
+                    help="record the decode queries and maintain the attention features (config 2: e.g. 128)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per launch of the dominant kernel")
     args = ap.parse_args()
