@@ -50,7 +50,7 @@ bool valid_config(const fkv_config *c) {
   if (c->budget < 1 || c->recent_keep < 0 || c->max_tokens_per_head < 1 || c->num_pages < 0) return false;
   if ((int64_t)c->num_layers * c->max_batch * c->num_kv_heads > (1 << 20)) return false;
   if (c->feature_window < 0 || c->feature_window % 8) return false;
-  if (c->feature_window && FeatSmem::bytes(c->head_dim, kFeatWarps, c->feature_window) > kMaxSmem) return false;
+  if (c->feature_window && FeatSmem::bytes(c->head_dim, 6 * c->group_size, kFeatWarps, c->feature_window) > kMaxSmem) return false;
   return true;
 }
 
@@ -186,7 +186,7 @@ void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float
 // Attention features of the segments on the work list (after a k_plan): grid (page groups, work items).
 template <int D>
 int launch_features_t(fkv_cache *c, int max_old, int nwork_bound, float scale_log2, cudaStream_t st) {
-  const size_t smem = FeatSmem::bytes(D, kFeatWarps, c->cfg.feature_window);
+  const size_t smem = FeatSmem::bytes(D, c->lay.F, kFeatWarps, c->cfg.feature_window);
   static size_t attr_bytes = 0;   // largest opt-in made so far
   if (smem > attr_bytes) {
     FKV_CUDA(cudaFuncSetAttribute(k_features<D, kFeatWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

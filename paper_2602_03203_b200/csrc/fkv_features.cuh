@@ -32,10 +32,10 @@ constexpr int kFeatPPW = 1;   // pages per warp
 struct FeatSmem {
   // K rows of the pages [nw * PPW][16][2D] | their meta rows [nw * PPW][16 * 49 words, padded] |
   // 2 x { queries of one head [W][2D] | M + log2 L [W] | pairs seen [W] }
-  static constexpr size_t kMeta = 16 * 49 * 4 + 64;   // room for the widest meta block (g = 8), 16-byte multiple
+  static __host__ __device__ size_t meta(int F) { return (size_t)kPage * (F + 1) * 4; }   // a multiple of 64 bytes
   static __host__ __device__ size_t qbuf(int D, int W) { return (size_t)W * 2 * D + (size_t)W * 8; }
-  static __host__ __device__ size_t bytes(int D, int nw, int W) {
-    return (size_t)nw * kFeatPPW * (2 * D * kPage + kMeta) + 2 * qbuf(D, W) + 16;
+  static __host__ __device__ size_t bytes(int D, int F, int nw, int W) {
+    return (size_t)nw * kFeatPPW * (2 * D * kPage + meta(F)) + 2 * qbuf(D, W) + 16;
   }
 };
 
@@ -69,8 +69,9 @@ __global__ void __launch_bounds__(NW * 32) k_features(Ctx c, float scale_log2) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
   const int gid = lane >> 2, tig = lane & 3;
   uint8_t *kpages = smem;
+  const size_t meta_bytes = FeatSmem::meta(c.F);
   uint8_t *metas = smem + (size_t)PG * PAGE_K;                     // the pages' meta blocks (features + positions)
-  uint8_t *qbuf0 = metas + (size_t)PG * FeatSmem::kMeta;           // two buffers of FeatSmem::qbuf bytes
+  uint8_t *qbuf0 = metas + (size_t)PG * meta_bytes;           // two buffers of FeatSmem::qbuf bytes
   const size_t qbytes = FeatSmem::qbuf(D, W);
   const int np = min(PG, npages - pg0);
 
@@ -85,7 +86,7 @@ __global__ void __launch_bounds__(NW * 32) k_features(Ctx c, float scale_log2) {
   for (int e = tid; e < np * meta_chunks; e += blockDim.x) {
     const int pg = e / meta_chunks, ch = e - pg * meta_chunks;
     const int pid = c.pt[(size_t)seg * c.max_pages + pg0 + pg];
-    cp_async16(smem_u32(metas + (size_t)pg * FeatSmem::kMeta + ch * 16), c.pool + (size_t)pid * c.page_bytes + c.off_f + ch * 16);
+    cp_async16(smem_u32(metas + (size_t)pg * meta_bytes + ch * 16), c.pool + (size_t)pid * c.page_bytes + c.off_f + ch * 16);
   }
   const uint8_t *hq = c.hist_q + (size_t)ls * W * Hq * D * 2;
   const float2 *hml = reinterpret_cast<const float2 *>(c.hist_ml) + (size_t)ls * W * Hq;
@@ -200,7 +201,7 @@ __global__ void __launch_bounds__(NW * 32) k_features(Ctx c, float scale_log2) {
         if (slot < n) {
           const float a8 = tig ? vals[1][0] : vals[0][0], a16 = tig ? vals[1][1] : vals[0][1];
           const float a32 = tig ? vals[1][2] : vals[0][2], all = tig ? vals[1][3] : vals[0][3];
-          float *f = reinterpret_cast<float *>(metas + (size_t)pg * FeatSmem::kMeta) + (slot % kPage) * (c.F + 1) + j * 6;
+          float *f = reinterpret_cast<float *>(metas + (size_t)pg * meta_bytes) + (slot % kPage) * (c.F + 1) + j * 6;
           const float chunk = all / (float)Lc;
           f[0] = a8 * (1.f / 8.f); f[1] = a16 * (1.f / 16.f); f[2] = a32 * (1.f / 32.f);
           f[3] = chunk;
@@ -216,7 +217,7 @@ __global__ void __launch_bounds__(NW * 32) k_features(Ctx c, float scale_log2) {
     const int pg = e / meta_chunks, ch = e - pg * meta_chunks;
     const int pid = c.pt[(size_t)seg * c.max_pages + pg0 + pg];
     *reinterpret_cast<uint4 *>(c.pool + (size_t)pid * c.page_bytes + c.off_f + ch * 16) =
-        *reinterpret_cast<const uint4 *>(metas + (size_t)pg * FeatSmem::kMeta + ch * 16);
+        *reinterpret_cast<const uint4 *>(metas + (size_t)pg * meta_bytes + ch * 16);
   }
 }
 
