@@ -79,7 +79,7 @@ typedef struct {
   int32_t num_pages;           /* pages in the pool; 0 = enough for every segment at capacity
                                   plus the transient copies of an all-layer eviction */
   int32_t feature_window;      /* W: decode queries kept on record per (layer, sequence) for the attention
-                                  features of Appendix B.1 (a multiple of 8; shared memory caps it, 352 for D = 128 and g = 4;
+                                  features of Appendix B.1 (a multiple of 8, at most 256;
                                   the paper's update length L, e.g. 256); 0 = the library does not
                                   maintain the features */
 } fkv_config;

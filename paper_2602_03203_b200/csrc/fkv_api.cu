@@ -30,7 +30,6 @@ thread_local std::string g_cuda_error;
 constexpr int kScorePPS = 8;  // consumer warps of the scorer = pages per tile
 constexpr int kAttendMinPages = 4;
 constexpr size_t kMaxSmem = 227 * 1024;
-constexpr int kFeatWarps = 8;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -50,7 +49,7 @@ bool valid_config(const fkv_config *c) {
   if (c->budget < 1 || c->recent_keep < 0 || c->max_tokens_per_head < 1 || c->num_pages < 0) return false;
   if ((int64_t)c->num_layers * c->max_batch * c->num_kv_heads > (1 << 20)) return false;
   if (c->feature_window < 0 || c->feature_window % 8) return false;
-  if (c->feature_window && FeatSmem::bytes(c->head_dim, 6 * c->group_size, kFeatWarps, c->feature_window) > kMaxSmem) return false;
+  if (c->feature_window > kFeatMaxQueries) return false;
   return true;
 }
 
@@ -183,19 +182,18 @@ void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float
 #undef FKV_SEL
 }
 
-// Attention features of the segments on the work list (after a k_plan): grid (page groups, work items).
+// Attention features of the segments on the work list (after a k_plan): grid (groups of 8 pages, work items).
 template <int D>
 int launch_features_t(fkv_cache *c, int max_old, int nwork_bound, float scale_log2, cudaStream_t st) {
-  const size_t smem = FeatSmem::bytes(D, c->lay.F, kFeatWarps, c->cfg.feature_window);
+  const size_t smem = FeatSmem::bytes(D, c->lay.F, c->cfg.feature_window);
   static size_t attr_bytes = 0;   // largest opt-in made so far
   if (smem > attr_bytes) {
-    FKV_CUDA(cudaFuncSetAttribute(k_features<D, kFeatWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    FKV_CUDA(cudaFuncSetAttribute(k_features<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     attr_bytes = smem;
   }
-  const int group = kFeatWarps * kFeatPPW;   // pages per CTA
-  dim3 grid(((max_old + kPage - 1) / kPage + group - 1) / group, nwork_bound);
+  dim3 grid(((max_old + kPage - 1) / kPage + kFeatPages - 1) / kFeatPages, nwork_bound);
   if (grid.x == 0 || grid.y == 0) return FKV_OK;
-  k_features<D, kFeatWarps><<<grid, kFeatWarps * 32, smem, st>>>(c->ctx, scale_log2);
+  k_features<D><<<grid, 256, smem, st>>>(c->ctx, scale_log2);
   FKV_LAUNCHED(c);
   return FKV_OK;
 }
