@@ -19,10 +19,11 @@
 //     padded query count, K = 16 per instruction) with shared-memory descriptors; the accumulator
 //     lives in tensor memory (one fp32 column per query), completion arrives on an mbarrier
 //     through tcgen05.commit;
-//   - four warps read the accumulator back with tcgen05.ld (lane = pair, 32 query columns at a
+//   - the warps read the accumulator back with tcgen05.ld (lane = pair, 32 query columns at a
 //     time); a thread owns ONE pair, and because the queries are ordered newest first the windows
-//     8 / 16 / 32 / all are running prefix sums along its row: exp2, mask, add - no reduction
-//     across threads;
+//     8 / 16 / 32 / all are running prefix sums along its row: exp2, (mask,) add.  Warps 0-3 take
+//     the newer half of the query axis, warps 4-7 the older half, whose sum they hand over
+//     through shared memory;
 //   - while a head is being multiplied and reduced, the next head's queries stream in.
 // The decode path pays 2 g D + 12 g bytes per token for the record instead of a read-modify-write
 // of every pair's feature row per token.
@@ -46,7 +47,7 @@ struct FeatSmem {
   // statistics: 2 x lq x (float M + log2 L, int pairs seen) | meta blocks of the 8 pages | barrier + tmem address
   static __host__ __device__ size_t bytes(int D, int F, int W) {
     const size_t need = 1024 + (size_t)(D / 64) * 128 * 128 + 2 * (size_t)(D / 64) * lq(W) * 128 + 2 * (size_t)lq(W) * 8 +
-                        kFeatPages * meta(F) + 64;
+                        kFeatPages * meta(F) + 64 + 128 * 4;   // + one float per pair: the older half's sum
     return need > 77 * 1024 ? need : 77 * 1024;   // never more than two CTAs per SM (tensor-memory budget)
   }
 };
@@ -132,6 +133,7 @@ __global__ void __launch_bounds__(256) k_features(Ctx c, float scale_log2) {
   uint8_t *metas = stats + 2 * (size_t)Lw * 8;
   uint64_t *bar = reinterpret_cast<uint64_t *>(metas + kFeatPages * meta_bytes);
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar + 1);
+  float *older = reinterpret_cast<float *>(smem + FeatSmem::bytes(D, c.F, W) - 1024 - 128 * 4);   // [128]: sums of the older half
 
   // Tensor memory: a power of two >= 32 columns that holds one fp32 column per query.
   uint32_t ncols = 32;
@@ -197,6 +199,8 @@ __global__ void __launch_bounds__(256) k_features(Ctx c, float scale_log2) {
   const uint32_t idesc = umma_idesc_bf16(ROWS, Lq);
   const int R = (warp & 3) * 32 + lane;              // epilogue: this thread's pair row of the tile
   const int slot = pg0 * kPage + R;
+  // Did every recorded query see the whole tile?  (The oldest one saw the fewest pairs.)
+  const bool whole = pg0 * kPage + ROWS <= hn[(cnt - Lc) % W];
   bool ok = true;
   uint32_t tmem_base = 0;
 
@@ -219,35 +223,55 @@ __global__ void __launch_bounds__(256) k_features(Ctx c, float scale_log2) {
       umma_commit(smem_u32(bar));
     }
     if (j + 1 < G) stage(j + 1, b ^ 1);              // streams in while head j is multiplied and reduced
-    if (warp < 4) {
-      // ---- epilogue: one pair per thread, its row of the accumulator, newest query first ----
+    {
+      // ---- epilogue: one pair per thread, its row of the accumulator, newest query first.  The query axis is
+      // split in two at a multiple of 32: warps 0-3 reduce [0, split), warps 4-7 [split, Lq). ----
       if (ok && !mbar_wait(smem_u32(bar), j & 1)) { set_status(c, kDevWaitTimeout); ok = false; }
       ok = __all_sync(0xffffffffu, ok);   // the tensor-memory loads below need the whole warp
       tc_fence_after();
+      const int split = Lq > 32 ? ((Lq / 2 + 31) & ~31) : Lq;
+      const int abeg = warp < 4 ? 0 : split, aend = warp < 4 ? split : Lq;
+      const float *sM = reinterpret_cast<const float *>(stats) + (size_t)b * Lw;
+      const int *sN = reinterpret_cast<const int *>(stats + 2 * (size_t)Lw * 4) + (size_t)b * Lw;
+      float run = 0.f, w8 = 0.f, w16 = 0.f, w32 = 0.f;
       if (ok) {
-        const float *sM = reinterpret_cast<const float *>(stats) + (size_t)b * Lw;
-        const int *sN = reinterpret_cast<const int *>(stats + 2 * (size_t)Lw * 4) + (size_t)b * Lw;
-        float run = 0.f, w8 = 0.f, w16 = 0.f, w32 = 0.f;
-        for (int a0 = 0; a0 < Lq; a0 += 32) {
+        for (int a0 = abeg; a0 < aend; a0 += 32) {
           if (a0 == 32) w32 = run;
           float v[32];
           tmem_ld32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)a0, v);
+          if (whole && a0 + 32 <= Lc) {              // every query of the chunk saw the whole tile: no masks
 #pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            if (i < 16 || a0 + i < Lq) {             // Lq is a multiple of 16: the second half of a chunk may be padding
+            for (int i = 0; i < 32; i += 4) {
               const float4 M4 = *reinterpret_cast<const float4 *>(sM + a0 + i);
-              const int4 N4 = *reinterpret_cast<const int4 *>(sN + a0 + i);
               if (i == 8 && a0 == 0) w8 = run;
               if (i == 16 && a0 == 0) w16 = run;
-              run += slot < N4.x ? ex2(v[i] * scale_log2 - M4.x) : 0.f;
-              run += slot < N4.y ? ex2(v[i + 1] * scale_log2 - M4.y) : 0.f;
-              run += slot < N4.z ? ex2(v[i + 2] * scale_log2 - M4.z) : 0.f;
-              run += slot < N4.w ? ex2(v[i + 3] * scale_log2 - M4.w) : 0.f;
+              run += (ex2(v[i] * scale_log2 - M4.x) + ex2(v[i + 1] * scale_log2 - M4.y)) +
+                     (ex2(v[i + 2] * scale_log2 - M4.z) + ex2(v[i + 3] * scale_log2 - M4.w));
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              if (i < 16 || a0 + i < Lq) {           // Lq is a multiple of 16: the second half of a chunk may be padding
+                const float4 M4 = *reinterpret_cast<const float4 *>(sM + a0 + i);
+                const int4 N4 = *reinterpret_cast<const int4 *>(sN + a0 + i);
+                if (i == 8 && a0 == 0) w8 = run;
+                if (i == 16 && a0 == 0) w16 = run;
+                run += slot < N4.x ? ex2(v[i] * scale_log2 - M4.x) : 0.f;
+                run += slot < N4.y ? ex2(v[i + 1] * scale_log2 - M4.y) : 0.f;
+                run += slot < N4.z ? ex2(v[i + 2] * scale_log2 - M4.z) : 0.f;
+                run += slot < N4.w ? ex2(v[i + 3] * scale_log2 - M4.w) : 0.f;
+              }
             }
           }
         }
-        if (Lq <= 16) w16 = run;
-        if (Lq <= 32) w32 = run;
+      }
+      tc_fence_before();
+      if (warp >= 4) older[R] = run;
+      asm volatile("bar.sync 1, 256;" ::: "memory");   // the older half's sums are in shared memory
+      if (warp < 4 && ok) {
+        if (split <= 16) w16 = run;   // windows wider than this thread's half (split is 16, or a multiple of 32)
+        if (split <= 32) w32 = run;
+        run += older[R];
         if (slot < n) {
           float *f = reinterpret_cast<float *>(metas + (size_t)(R / kPage) * meta_bytes) + (R % kPage) * (c.F + 1) + j * 6;
           const float chunk = run / (float)Lc;
@@ -257,7 +281,6 @@ __global__ void __launch_bounds__(256) k_features(Ctx c, float scale_log2) {
           f[5] = fmaf(kFeatDecay, f[5], chunk);
         }
       }
-      tc_fence_before();
     }
   }
   // ---- the refreshed meta blocks go back to their page records (every row was written by one thread) ----
