@@ -145,14 +145,20 @@ __global__ void __launch_bounds__(256) k_features(Ctx c, float scale_log2) {
   }
 
   // ---- A: the K rows of this group's pages, chunk for chunk (row pitch 128 B per 64-channel half) ----
-  for (int e = tid; e < ROWS * NCH; e += blockDim.x) {
-    const int R = e / NCH, ch = e - R * NCH, pg = R / kPage, r = R - pg * kPage;
-    uint8_t *dst = At + (size_t)(ch >> 3) * ROWS * 128 + (size_t)R * 128 + (ch & 7) * 16;
-    if (pg < np) {
-      const int pid = c.pt[(size_t)seg * c.max_pages + pg0 + pg];
-      cp_async16(smem_u32(dst), c.pool + (size_t)pid * c.page_bytes + (size_t)r * 4 * D + ch * 16);
-    } else {
-      *reinterpret_cast<uint4 *>(dst) = make_uint4(0u, 0u, 0u, 0u);
+  {
+    // Thread = one 16-byte chunk column (ch) of rows R0, R0 + 256 / NCH, ...: fixed offsets, a pointer per page.
+    constexpr int RSTEP = 256 / NCH;
+    const int ch = tid % NCH, R0 = tid / NCH;
+    const uint32_t dst0 = smem_u32(At) + (uint32_t)((ch >> 3) * ROWS * 128 + (ch & 7) * 16);
+    const int *ptrow = c.pt + (size_t)seg * c.max_pages + pg0;
+#pragma unroll
+    for (int k = 0; k < ROWS / RSTEP; ++k) {
+      const int Rr = R0 + k * RSTEP, pg = Rr / kPage, r = Rr % kPage;
+      if (pg < np)
+        cp_async16(dst0 + Rr * 128, c.pool + (size_t)ptrow[pg] * c.page_bytes + r * 4 * D + ch * 16);
+      else
+        *reinterpret_cast<uint4 *>(At + (size_t)(ch >> 3) * ROWS * 128 + (size_t)Rr * 128 + (ch & 7) * 16) =
+            make_uint4(0u, 0u, 0u, 0u);
     }
   }
   const int meta_chunks = (int)(meta_bytes / 16);
@@ -173,14 +179,20 @@ __global__ void __launch_bounds__(256) k_features(Ctx c, float scale_log2) {
     uint8_t *qs = Qt + (size_t)b * qbuf;
     float *sM = reinterpret_cast<float *>(stats) + (size_t)b * Lw;
     int *sN = reinterpret_cast<int *>(stats + 2 * (size_t)Lw * 4) + (size_t)b * Lw;
-    for (int e = tid; e < Lq * NCH; e += blockDim.x) {
-      const int a = e / NCH, ch = e - a * NCH;
-      uint8_t *dst = qs + (size_t)(ch >> 3) * Lw * 128 + (size_t)a * 128 + (((ch & 7) ^ (a & 7)) << 4);
-      if (a < Lc) {
-        const int hs = newest - a + (newest < a ? W : 0);
-        cp_async16(smem_u32(dst), hq + ((size_t)hs * Hq + qh) * D * 2 + ch * 16);
-      } else {
-        *reinterpret_cast<uint4 *>(dst) = make_uint4(0u, 0u, 0u, 0u);
+    {
+      constexpr int RSTEP = 256 / NCH;
+      const int ch = tid % NCH;
+      uint8_t *col = qs + (size_t)(ch >> 3) * Lw * 128;
+      const uint8_t *src0 = hq + (size_t)qh * D * 2 + ch * 16;
+      const size_t hstride = (size_t)Hq * D * 2;
+      for (int a = tid / NCH; a < Lq; a += RSTEP) {
+        uint8_t *dst = col + (size_t)a * 128 + (((ch & 7) ^ (a & 7)) << 4);
+        if (a < Lc) {
+          const int hs = newest - a + (newest < a ? W : 0);
+          cp_async16(smem_u32(dst), src0 + hs * hstride);
+        } else {
+          *reinterpret_cast<uint4 *>(dst) = make_uint4(0u, 0u, 0u, 0u);
+        }
       }
     }
     for (int a = tid; a < Lq; a += blockDim.x) {
