@@ -93,6 +93,19 @@ def select_sampled(phi, B, R, noise):
     return kept[:nk].copy(), cand[:ncand.value].copy()
 
 
+H2O_COLUMN, SNAPKV_COLUMN = 4, 0
+
+
+def score_feature(A, g, column):
+    """Baseline score (H2O: column 4, SnapKV: column 0): mean over the g heads of one feature column, fp32."""
+    A, pA = _c(A, np.float32)
+    n = A.shape[0]
+    assert A.shape == (n, 6 * g) and 0 <= column < 6
+    phi = np.empty(n, np.float32)
+    lib().fkv_oracle_score_feature(pA, n, int(g), int(column), phi.ctypes.data_as(ctypes.c_void_p))
+    return phi
+
+
 def features(K, q, nvalid, A, scale=None, decay=0.9):
     """Attention features refreshed at the end of a chunk (Appendix B.1).
 

@@ -221,6 +221,22 @@ void fkv_oracle_attend(const uint16_t *q, const uint16_t *K, const uint16_t *V, 
 }
 
 /*
+ * Baseline scores of Appendix E.2 that need no learned scorer: one attention-feature column, pooled
+ * (averaged, as the paper pools over a group elsewhere) over the g query heads of the KV head:
+ *   H2O    "cumulative attention scores"                         -> the direct-sum column (4)
+ *   SnapKV "the attention scores of the final 8 tokens"          -> the window-8 column (0)
+ * The sum runs over the heads in order and is divided by g, all in fp32 (the precision the ranking
+ * is decided in).  A: [n][6g]; phi: [n].
+ */
+void fkv_oracle_score_feature(const float *A, int n, int g, int column, float *phi) {
+  for (int i = 0; i < n; ++i) {
+    float acc = 0.0f;
+    for (int j = 0; j < g; ++j) acc = acc + A[(size_t)i * 6 * g + (size_t)j * 6 + column];
+    phi[i] = acc / (float)g;
+  }
+}
+
+/*
  * Attention features of Appendix B.1 for one segment, refreshed at an eviction that closes a chunk
  * of nq decode queries (chronological order, the last one the most recent).  Query t of query head j
  * attended the first nvalid[t] pairs (the cache as it was then); its probabilities are

@@ -445,3 +445,21 @@ def test_features_chunks_accumulate_and_decay():
     assert np.allclose(A2[:, 5::6], 0.9 * c1 + c2, atol=1e-6)           # per-chunk decay 0.9
     assert np.allclose(A2[:, 3::6], c2, atol=1e-7)                      # window features belong to the last chunk only
     assert np.allclose(A2[:, 3::6].sum(0), 1.0, atol=1e-5)              # mean of probability rows still sums to 1
+
+
+# ---------------------------------------------------------------- baseline scores (Appendix E.2: H2O, SnapKV)
+def test_feature_column_scores():
+    rng = np.random.default_rng(21)
+    n, g = 40, 4
+    A = rng.random((n, 6 * g)).astype(np.float32)
+    for col in range(6):
+        phi = oracle.score_feature(A, g, col)
+        assert np.allclose(phi, A.reshape(n, g, 6)[:, :, col].astype(np.float64).mean(1), rtol=1e-6)
+    # one head only: the column itself; a head-major layout mistake (6 heads x g columns) fails here
+    A1 = np.zeros((3, 6 * g), np.float32); A1[1, 2 * 6 + 4] = 8.0          # head 2, direct-sum column
+    assert oracle.score_feature(A1, g, oracle.H2O_COLUMN).tolist() == [0.0, 2.0, 0.0]
+    assert oracle.score_feature(A1, g, oracle.SNAPKV_COLUMN).tolist() == [0.0, 0.0, 0.0]
+    # H2O keeps the pairs with the highest cumulative attention: selection on that column
+    cum = np.array([5, 1, 4, 2, 3], np.float32)
+    A2 = np.zeros((5, 6), np.float32); A2[:, 4] = cum
+    assert oracle.select(oracle.score_feature(A2, 1, oracle.H2O_COLUMN), 3, 0).tolist() == [0, 2, 4]
