@@ -166,6 +166,22 @@ int fkv_evict(fkv_cache *c, int layer, void *stream);
 int fkv_evict_sampled(fkv_cache *c, int layer, const float *noise, int32_t noise_stride, void *stream);
 
 /*
+ * evict(layer) with a BASELINE score in place of the learned scorer - Appendix E.2.  The score of a
+ * pair is one column of its attention features, averaged over the g query heads of the KV head
+ * (summed in head order, divided by g, fp32): column FKV_FEATURE_CUM_SUM is H2O (cumulative
+ * attention), FKV_FEATURE_WINDOW8 is SnapKV as the paper uses it (attention of the final 8 tokens).
+ * Selection, compaction and (with a feature window) the feature refresh are those of fkv_evict; no
+ * scorer needs to be loaded.  R-KV's redundancy term is not provided.
+ */
+#define FKV_FEATURE_WINDOW8 0
+#define FKV_FEATURE_WINDOW16 1
+#define FKV_FEATURE_WINDOW32 2
+#define FKV_FEATURE_WINDOW_CHUNK 3
+#define FKV_FEATURE_CUM_SUM 4
+#define FKV_FEATURE_CUM_DECAY 5
+int fkv_evict_by_feature(fkv_cache *c, int layer, int32_t column, void *stream);
+
+/*
  * decode_attn(q) - Appendix A: out[s][h] = sum_i softmax_i(scale <q[s][h], k_i>) v_i
  * over all retained pairs i of the KV head that query head h belongs to
  * (h / g).  q, out: dev [max_batch][Hkv*g][D] bf16.  scale 0 means 1/sqrt(D).

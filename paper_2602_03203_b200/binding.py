@@ -26,7 +26,7 @@ EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", 
            "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
            "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
            "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing",
-           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled", "fkv_update_features"]
+           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled", "fkv_update_features", "fkv_evict_by_feature"]
 
 
 class FkvConfig(ctypes.Structure):
@@ -148,6 +148,10 @@ class Cache:
         """The paper's sampled action; noise [layers of the call][batch][Hkv][stride] standard Gumbel draws."""
         _check(lib().fkv_evict_sampled(self._h, layer, _ptr(noise, torch.float32), int(noise.shape[-1]), _stream()),
                "fkv_evict_sampled")
+
+    def evict_by_feature(self, column, layer=ALL_LAYERS):
+        """Baseline eviction: score = one feature column (4: H2O cumulative attention, 0: SnapKV last-8 window)."""
+        _check(lib().fkv_evict_by_feature(self._h, layer, int(column), _stream()), "fkv_evict_by_feature")
 
     def decode_attn(self, layer, q, out=None, scale=0.0):
         if out is None:

@@ -466,7 +466,7 @@ static int sampled_candidates(int n, int B, int R) {
   return std::min(2 * (n - B), n - std::min(R, B));
 }
 
-static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_stride, void *stream) {
+static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_stride, int feature_column, void *stream) {
   if (!c || (layer != FKV_ALL_LAYERS && !layer_ok(c, layer))) return FKV_ERR_INVALID_ARG;
   const int l0 = layer == FKV_ALL_LAYERS ? 0 : layer, l1 = layer == FKV_ALL_LAYERS ? c->cfg.num_layers : layer + 1;
   const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
@@ -476,7 +476,7 @@ static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_str
     for (int s = 0; s < batch; ++s) {
       const int n = c->h_len[(size_t)l * batch + s], B = c->h_budget[s];
       if (n > B) {
-        for (int h = 0; h < Hkv; ++h)
+        for (int h = 0; h < Hkv && feature_column < 0; ++h)
           if (!c->loaded[(size_t)l * Hkv + h]) return FKV_ERR_NOT_READY;
         if (noise && sampled_candidates(n, B, c->cfg.recent_keep) > noise_stride) return FKV_ERR_INVALID_ARG;
         nactive += Hkv;
@@ -497,7 +497,13 @@ static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_str
     if (rcf) return rcf;
   }
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[1], st));
-  int rc = launch_score_any(c, c->ctx.scores, 0, (int)std::min<long long>(tiles, 1 << 30), st);
+  int rc = FKV_OK;
+  if (feature_column < 0) {
+    rc = launch_score_any(c, c->ctx.scores, 0, (int)std::min<long long>(tiles, 1 << 30), st);
+  } else {   // a baseline: the score is a feature column
+    k_score_feature<<<dim3((max_old + 127) / 128, nactive), 128, 0, st>>>(c->ctx, c->ctx.scores, 0, feature_column);
+    FKV_LAUNCHED(c);
+  }
   if (rc) return rc;
   if (tm) FKV_CUDA(cudaEventRecord(c->ev[2], st));
   if (noise) {   // sampled action: scores -> keep-priorities (in place), then the same selection over them
@@ -525,11 +531,16 @@ static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_str
   return FKV_OK;
 }
 
-int fkv_evict(fkv_cache *c, int layer, void *stream) { return evict_impl(c, layer, nullptr, 0, stream); }
+int fkv_evict(fkv_cache *c, int layer, void *stream) { return evict_impl(c, layer, nullptr, 0, -1, stream); }
+
+int fkv_evict_by_feature(fkv_cache *c, int layer, int32_t column, void *stream) {
+  if (column < 0 || column > 5) return FKV_ERR_INVALID_ARG;
+  return evict_impl(c, layer, nullptr, 0, column, stream);
+}
 
 int fkv_evict_sampled(fkv_cache *c, int layer, const float *noise, int32_t noise_stride, void *stream) {
   if (!noise || noise_stride < 1) return FKV_ERR_INVALID_ARG;
-  return evict_impl(c, layer, noise, noise_stride, stream);
+  return evict_impl(c, layer, noise, noise_stride, -1, stream);
 }
 
 int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream) {

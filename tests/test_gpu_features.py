@@ -116,3 +116,63 @@ def test_decode_evict_cycle_with_maintained_features():
             assert np.all(np.abs(got - A1[kept_g]) <= FEAT_ATOL + FEAT_RTOL * np.abs(A1[kept_g]))
             st[h] = dict(K=d["K"][kept_g], V=d["V"][kept_g], A=got.copy(), pos=d["pos"][kept_g])   # follow the GPU's state
     assert c.device_status()[0] == 0
+
+
+@pytest.mark.parametrize("column", [oracle.H2O_COLUMN, oracle.SNAPKV_COLUMN])
+def test_baseline_eviction_on_maintained_features(column):
+    # H2O / SnapKV (Appendix E.2) on the library's own features: a chunk of decoding, then an eviction
+    # whose score is a feature column.  No scorer is loaded.  The kept set follows from the refreshed
+    # features the library exports; those features are checked against the oracle's.
+    B, Lev = 96, 32
+    w = wl.Workload("base", 1, 2, 4, 128, (B, 70), (B, B), 8, 54, "normal")
+    c = binding.from_workload(w, feature_window=Lev)
+    st = {}
+    for s in range(2):
+        K, V, A, pos = wl.layer_inputs(w, 0, s)
+        c.prefill(0, s, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
+        for h in range(2):
+            st[(s, h)] = dict(K=bits(K)[h], A=npf(A)[h].copy(), q=[], nv=[])
+    g = w.group_size
+    for step in range(Lev):
+        k, v = wl.new_kv(w, 0, step); q = wl.queries(w, 0, step)
+        c.append_decode_attn(0, k.cuda(), v.cuda(), q.cuda())
+        for (s, h), d in st.items():
+            d["K"] = np.concatenate([d["K"], bits(k)[s, h][None]])
+            d["A"] = np.concatenate([d["A"], np.zeros((1, 6 * g), np.float32)])
+            d["q"].append(bits(q)[s, h * g:(h + 1) * g]); d["nv"].append(len(d["K"]))
+    c.update_features(0)
+    feats = {key: npf(c.export_head(0, key[0], key[1])[2]) for key in st}
+    c.evict_by_feature(column, 0)
+    assert c.lengths(0) == [B, B]
+    for (s, h), d in st.items():
+        exp = oracle.features(d["K"], np.stack(d["q"]), np.array(d["nv"], np.int32), d["A"])
+        assert np.all(np.abs(feats[(s, h)] - exp) <= FEAT_ATOL + FEAT_RTOL * np.abs(exp))
+        n = len(d["K"])
+        # NOTE the eviction refreshes the features once more (the chunk is still open after update_features):
+        # window columns are recomputed (same values), the cumulative columns move again.
+        again = oracle.features(d["K"], np.stack(d["q"]), np.array(d["nv"], np.int32), feats[(s, h)])
+        _, _, a2, p2 = c.export_head(0, s, h)
+        kept = oracle.select(oracle.score_feature(again, g, column), B, 8)
+        phi = oracle.score_feature(again, g, column)
+        assert kept_set_within_band(phi, kept, npf(p2), n, B, 8, 1e-5)
+        assert npf(p2)[-8:].tolist() == list(range(n - 8, n))
+    assert c.device_status()[0] == 0
+
+
+def test_baseline_eviction_bit_exact_on_given_features():
+    # With the features given (no window), the baseline score is a pure function of the stored rows:
+    # the kept list must equal the oracle's, bit for bit.
+    w = wl.Workload("base2", 2, 2, 7, 64, (500, 333), (200, 100), 16, 55, "normal")
+    c = binding.from_workload(w)
+    hold = {}
+    for l in range(2):
+        for s in range(2):
+            K, V, A, pos = wl.layer_inputs(w, l, s)
+            c.prefill(l, s, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
+            hold[(l, s)] = npf(A)
+    c.evict_by_feature(oracle.H2O_COLUMN)
+    for (l, s), A in hold.items():
+        for h in range(2):
+            kept = oracle.select(oracle.score_feature(A[h], 7, oracle.H2O_COLUMN), w.budgets[s], 16)
+            assert np.array_equal(npf(c.export_head(l, s, h)[3]), kept)
+    assert c.device_status()[0] == 0
