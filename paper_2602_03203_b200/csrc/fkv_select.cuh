@@ -22,8 +22,8 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-constexpr int kSelThreads = 1024;
-constexpr int kSelBins = 2048;
+constexpr int kSelThreads = 1024;   // the large variant: 1024 threads x 32 keys = one round of 32768
+constexpr int kSelSmallThreads = 512, kSelSmallPerThread = 16;   // segments of <= 8192 competing pairs: two CTAs per SM
 
 // Fresh page ids of one compacted segment: copied from the batch the planner
 // reserved at the top of the free stack into the segment's row of pt_new.
@@ -60,18 +60,20 @@ __global__ void k_fill_pt_new(Ctx c, int seg0, int nseg) {
 // slot order, g_j the caller's standard Gumbel draw.  Keeping the best m - E priorities (a MODE 0
 // pass over them) then evicts exactly the E candidates with the largest -score + g: E draws
 // without replacement from softmax(-score) over the candidates.  prio may be the scores array.
-constexpr int kSelPerThread = 32;
-constexpr int kSelRound = kSelThreads * kSelPerThread;
+constexpr int kSelRound = kSelThreads * 32;   // keys one CTA of the large variant holds in registers
 
 // Score back from its ordering key (canonical: -0 came in as +0, NaN as -infinity).
 __device__ __forceinline__ float key_score(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-template <bool SINGLE, int MODE>
-__global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scores, int32_t *idx, int32_t *kept_count,
+template <bool SINGLE, int MODE, int THREADS, int PER>
+__global__ void __launch_bounds__(THREADS) k_select(Ctx c, const float *scores, int32_t *idx, int32_t *kept_count,
                                                          int seg_base, int fill_pages, float *prio,
                                                          const float *noise, int noise_stride, int noise_base) {
+  constexpr int kSelBins = 2 * THREADS, kSelPerThread = PER, kSelRound = THREADS * PER, NWARPS = THREADS / 32;
+  constexpr int kLogBins = THREADS == 1024 ? 11 : THREADS == 512 ? 10 : 9;
+  static_assert(THREADS == 1024 || THREADS == 512 || THREADS == 256, "bins = 2 x threads, a power of two");
   __shared__ unsigned s_hist[kSelBins];
   __shared__ int s_scan[33];
   __shared__ unsigned s_red[64];
@@ -91,19 +93,19 @@ __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scor
   if (MODE == 0) {
     if (kept_count && tid == 0) kept_count[seg - seg_base] = p.n_new;
     // The protected recent slots close the list.
-    for (int j = tid; j < p.r; j += kSelThreads) out[k + j] = m + j;
+    for (int j = tid; j < p.r; j += THREADS) out[k + j] = m + j;
     if (k <= 0) return;
     if (k >= m) {
-      for (int j = tid; j < m; j += kSelThreads) out[j] = j;
+      for (int j = tid; j < m; j += THREADS) out[j] = j;
       return;
     }
   } else {
     if (k <= 0) {   // every competing pair is a candidate: rank = slot
-      for (int j = tid; j < m; j += kSelThreads) pr[j] = key_score(score_key(sc[j])) - nz[j];
+      for (int j = tid; j < m; j += THREADS) pr[j] = key_score(score_key(sc[j])) - nz[j];
       return;
     }
     if (k >= m) {   // nothing to evict
-      for (int j = tid; j < m; j += kSelThreads) pr[j] = INFINITY;
+      for (int j = tid; j < m; j += THREADS) pr[j] = INFINITY;
       return;
     }
   }
@@ -137,8 +139,8 @@ __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scor
   kmax = __reduce_max_sync(0xffffffffu, kmax);
   if (lane == 0) { s_red[warp] = kmin; s_red[32 + warp] = kmax; }
   __syncthreads();
-  kmin = __reduce_min_sync(0xffffffffu, s_red[lane]);
-  kmax = __reduce_max_sync(0xffffffffu, s_red[32 + lane]);
+  kmin = __reduce_min_sync(0xffffffffu, lane < NWARPS ? s_red[lane] : 0xffffffffu);
+  kmax = __reduce_max_sync(0xffffffffu, lane < NWARPS ? s_red[32 + lane] : 0u);
 
   uint32_t T = kmin;
   unsigned need = (unsigned)k;
@@ -147,8 +149,8 @@ __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scor
     unsigned krem = (unsigned)k;
     int bits = 32 - __clz(wmax);
     for (;;) {
-      const int shift = bits > 11 ? bits - 11 : 0;
-      for (int b = tid; b < kSelBins; b += kSelThreads) s_hist[b] = 0;
+      const int shift = bits > kLogBins ? bits - kLogBins : 0;
+      for (int b = tid; b < kSelBins; b += THREADS) s_hist[b] = 0;
       __syncthreads();
       for (int round = 0; round < rounds; ++round) {
         if (!SINGLE) load_round(round);
@@ -203,7 +205,7 @@ __global__ void __launch_bounds__(kSelThreads) k_select(Ctx c, const float *scor
     if (lane == 31) s_wsum[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-      unsigned long long w = s_wsum[lane], winc = w;
+      unsigned long long w = lane < NWARPS ? s_wsum[lane] : 0ull, winc = w;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         unsigned long long t = __shfl_up_sync(0xffffffffu, winc, o);
