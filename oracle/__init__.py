@@ -106,6 +106,33 @@ def score_feature(A, g, column):
     return phi
 
 
+def golden(A, B, L):
+    """Golden Eviction labels of one attention group.  A: [g][T][T] fp32 attention probabilities.
+
+    Returns (alpha [M][T] future scores, kept [M][B - L] retained positions per eviction step).
+    """
+    A, pA = _c(A, np.float32)
+    g, T, T2 = A.shape
+    assert T == T2 and 0 < L < B
+    M = max(0, (T - B + L - 1) // L - 1)
+    alpha = np.zeros((max(M, 1), T), np.float32)
+    kept = np.zeros((max(M, 1), B - L), np.int32)
+    lib().fkv_oracle_golden.restype = ctypes.c_int
+    m = lib().fkv_oracle_golden(pA, g, T, int(B), int(L), alpha.ctypes.data_as(ctypes.c_void_p),
+                                kept.ctypes.data_as(ctypes.c_void_p))
+    assert m == M
+    return alpha[:M], kept[:M]
+
+
+def golden_select(alpha, B, L):
+    """Retained sets [M][B - L] of Golden Eviction from given future scores alpha [M][T]."""
+    alpha, pa = _c(alpha, np.float32)
+    M, T = alpha.shape
+    kept = np.zeros((M, B - L), np.int32)
+    lib().fkv_oracle_golden_select(pa, T, int(B), int(L), M, kept.ctypes.data_as(ctypes.c_void_p))
+    return kept
+
+
 def features(K, q, nvalid, A, scale=None, decay=0.9):
     """Attention features refreshed at the end of a chunk (Appendix B.1).
 

@@ -286,6 +286,57 @@ void fkv_oracle_features(const uint16_t *K, int n, int D, int g, const uint16_t 
 }
 
 /*
+ * The retained sets of Golden Eviction from given future scores alpha [M][T] (Eq. 5, second half):
+ * step t prunes the B cached pairs - the B - L retained at step t - 1 plus the L tokens that just left
+ * the recent window; [0, B) at step 1 - to the B - L with the largest alpha[t][.]; ties: lower position.
+ */
+void fkv_oracle_golden_select(const float *alpha, int T, int B, int L, int M, int32_t *kept) {
+  int32_t *cache = (int32_t *)malloc((size_t)B * sizeof(int32_t));
+  ranked_t *order = (ranked_t *)malloc((size_t)B * sizeof(ranked_t));
+  for (int i = 0; i < B; ++i) cache[i] = i;
+  for (int t = 1; t <= M; ++t) {
+    for (int j = 0; j < B; ++j) { order[j].score = canonical(alpha[(size_t)(t - 1) * T + cache[j]]); order[j].slot = cache[j]; }
+    qsort(order, (size_t)B, sizeof(ranked_t), by_score_then_slot);
+    int32_t *out = kept + (size_t)(t - 1) * (B - L);
+    for (int j = 0; j < B - L; ++j) out[j] = order[j].slot;
+    qsort(out, (size_t)(B - L), sizeof(int32_t), by_slot);
+    for (int j = 0; j < B - L; ++j) cache[j] = out[j];
+    for (int j = 0; j < L; ++j) cache[B - L + j] = B + (t - 1) * L + j;   /* the tokens that leave the recent window next */
+  }
+  free(cache); free(order);
+}
+
+/*
+ * Golden Eviction labels (Section 3.2, Eq. 3-5) for one attention group.
+ * A: [g][T][T] attention probabilities of the g heads (row = query position, column = key position).
+ * Blocks of L query rows start at the first eviction position B + L: block t = rows
+ * [B + t L, B + (t + 1) L), t = 1 .. M, M = ceil((T - B) / L) - 1; the last block is zero-padded to L rows.
+ *   block score   a~_t[i]  = average over the g heads and the L rows of the block of A[h][r][i]   (Eq. 3, 4)
+ *   future score  alpha[t][i] = max over j in [t, M] of a~_j[i]                                   (Eq. 5)
+ *   retained set  s_t = Top_{B-L}(alpha[t][.]) over the pairs still cached: s_0 = [0, B); at step t the
+ *                 cache holds s_{t-1} ... as B pairs: the B - L retained at step t - 1 plus the L tokens
+ *                 [B + (t-2) L, B + (t-1) L) that just left the recent window (for t = 1: [0, B)); the
+ *                 L newest tokens are kept regardless and are not listed.  Ties: lower position first.
+ * alpha: [M][T] out (row t - 1 is step t); kept: [M][B - L] out, ascending positions.  Returns M.
+ */
+int fkv_oracle_golden(const float *A, int g, int T, int B, int L, float *alpha, int32_t *kept) {
+  int M = (T - B + L - 1) / L - 1;
+  if (M < 1) return 0;
+  for (int t = 1; t <= M; ++t)
+    for (int i = 0; i < T; ++i) {
+      double acc = 0.0;
+      for (int h = 0; h < g; ++h)
+        for (int r = B + t * L; r < B + (t + 1) * L && r < T; ++r) acc += (double)A[((size_t)h * T + r) * T + i];
+      alpha[(size_t)(t - 1) * T + i] = (float)(acc / ((double)g * (double)L));
+    }
+  for (int t = M - 1; t >= 1; --t)
+    for (int i = 0; i < T; ++i)
+      if (alpha[(size_t)t * T + i] > alpha[(size_t)(t - 1) * T + i]) alpha[(size_t)(t - 1) * T + i] = alpha[(size_t)t * T + i];
+  fkv_oracle_golden_select(alpha, T, B, L, M, kept);
+  return M;
+}
+
+/*
  * One eviction step over many independent segments (score -> select ->
  * compact), the unit the CPU baseline times.  Segment i has n[i] pairs laid
  * out densely from offset off[i] (in pairs) in K, V, A, pos and phi; the

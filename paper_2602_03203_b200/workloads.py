@@ -214,6 +214,21 @@ def gumbel_noise(w: Workload, layer: int, stride: int, event: int = 0, device="c
     return (-torch.log(-torch.log(u))).to(torch.float32).contiguous()
 
 
+def causal_attention(seed: int, g: int, T: int, device="cpu", heavy: int = 8) -> torch.Tensor:
+    """Synthetic causal attention probabilities [g][T][T] fp32 (rows sum to 1) for the Golden-Eviction
+    label builder: random logits, a few "heavy hitter" key positions that many queries attend to, and a
+    recency bias - the patterns the paper's Figure 1 describes.  Input data only."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(0x5EED0000 + seed)
+    logits = torch.randn((g, T, T), generator=gen, device=device)
+    hh = torch.randperm(T, generator=gen, device=device)[:heavy]
+    logits[:, :, hh] += 3.0
+    r = torch.arange(T, device=device)
+    logits = logits - 0.002 * (r.view(1, T, 1) - r.view(1, 1, T)).clamp(min=0)
+    logits = logits.masked_fill(r.view(1, 1, T) > r.view(1, T, 1), float("-inf"))
+    return torch.softmax(logits, dim=-1).contiguous()
+
+
 def segment_list(w: Workload) -> List[Tuple[int, int, int]]:
     """All (layer, seq, kv_head) segments of a workload."""
     return [(l, s, h) for l in range(w.num_layers) for s in range(w.batch) for h in range(w.num_kv_heads)]

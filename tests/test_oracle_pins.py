@@ -463,3 +463,66 @@ def test_feature_column_scores():
     cum = np.array([5, 1, 4, 2, 3], np.float32)
     A2 = np.zeros((5, 6), np.float32); A2[:, 4] = cum
     assert oracle.select(oracle.score_feature(A2, 1, oracle.H2O_COLUMN), 3, 0).tolist() == [0, 2, 4]
+
+
+# ---------------------------------------------------------------- Golden Eviction labels (Section 3.2, Eq. 3-5)
+def _golden_brute(A, B, L):
+    """Independent statement with numpy slicing and Python sets (not the oracle's loops)."""
+    g, T, _ = A.shape
+    M = math.ceil((T - B) / L) - 1
+    blocks = np.zeros((M, T))
+    for t in range(1, M + 1):
+        rows = A[:, B + t * L:min(T, B + (t + 1) * L), :].astype(np.float64)
+        blocks[t - 1] = rows.sum(axis=(0, 1)) / (g * L)
+    alpha = np.maximum.accumulate(blocks[::-1], axis=0)[::-1]
+    cache, kept = list(range(B)), []
+    for t in range(1, M + 1):
+        a32 = alpha[t - 1].astype(np.float32)
+        best = sorted(cache, key=lambda i: (-a32[i], i))[:B - L]
+        kept.append(sorted(best))
+        cache = sorted(best) + list(range(B + (t - 1) * L, B + t * L))
+    return alpha, np.array(kept, np.int32)
+
+
+def test_golden_against_brute_force_and_invariants():
+    for seed, (g, T, B, L) in enumerate([(2, 96, 32, 8), (4, 130, 40, 16), (1, 64, 24, 8), (3, 77, 30, 10)]):
+        A = wl.causal_attention(seed, g, T).numpy()
+        alpha, kept = oracle.golden(A, B, L)
+        M = math.ceil((T - B) / L) - 1                                   # the paper's count of eviction steps
+        assert alpha.shape == (M, T) and kept.shape == (M, B - L)
+        a_ref, k_ref = _golden_brute(A, B, L)
+        assert np.allclose(alpha, a_ref, rtol=1e-6, atol=1e-9) and np.array_equal(kept, k_ref)
+        assert np.all(alpha[:-1] >= alpha[1:])                            # a maximum over fewer future blocks
+        cache = set(range(B))
+        for t in range(M):
+            assert np.all(np.diff(kept[t]) > 0) and set(kept[t].tolist()) <= cache   # evictions are irreversible
+            cache = set(kept[t].tolist()) | set(range(B + t * L, B + (t + 1) * L))
+
+
+def test_golden_closed_forms():
+    # Every query puts 60 % of its attention on key 5 and spreads the rest evenly over what it can see:
+    # key 5 has the top future score at every step and is always retained; the others tie, so the
+    # lowest positions survive.
+    g, T, B, L = 2, 80, 24, 8
+    A = np.zeros((g, T, T), np.float32)
+    for r in range(T):
+        if r >= 5:
+            A[:, r, :r + 1] = 0.4 / r if r > 0 else 0.0
+            A[:, r, 5] = 0.6
+        else:
+            A[:, r, :r + 1] = 1.0 / (r + 1)
+    alpha, kept = oracle.golden(A, B, L)
+    M = math.ceil((T - B) / L) - 1
+    assert M == 6
+    assert np.all(np.argmax(alpha, axis=1) == 5) and np.allclose(alpha[:, 5], 0.6)
+    for t in range(M):
+        assert 5 in kept[t]
+    # block t averages 0.4 / r over its rows: decreasing in t, so the future score IS the block score
+    t = 2
+    rows = np.arange(B + t * L, B + (t + 1) * L)
+    assert np.isclose(alpha[t - 1, 0], np.mean(0.4 / rows), rtol=1e-5)
+    # the last block is zero-padded to L rows when T is not on a block boundary
+    A2 = A[:, :76, :76]
+    alpha2, _ = oracle.golden(A2, B, L)
+    rows = np.arange(B + 6 * L, 76)
+    assert np.isclose(alpha2[5, 0], np.sum(0.4 / rows) / L, rtol=1e-5)
