@@ -322,6 +322,27 @@ int fkv_launch_count(const fkv_cache *c, uint64_t *launches);
 int fkv_decode_attn_dense_noalloc(const void *q, const void *k, const void *v, int32_t n, int32_t num_kv_heads,
                                   int32_t group_size, int32_t head_dim, float scale, void *out, void *stream);
 
+/*
+ * Golden Eviction labels - Section 3.2, Eq. 3-5: the supervision targets of the scorer, from the full
+ * attention matrix of ONE attention group (no cache handle involved).
+ *   attn: dev fp32 [g][T][T] attention probabilities of the group's g heads, row = query position,
+ *         column = key position.
+ * Query rows are cut into blocks of L starting at the first eviction position B + L (the last block
+ * zero-padded): M = ceil((T - B) / L) - 1 blocks = eviction steps (fkv_golden_steps).  Block score =
+ * average over the g heads and the block's L rows; future score alpha[t][i] = maximum of the block
+ * scores of pair i over blocks t .. M; retained set of step t = the B - L pairs with the largest
+ * alpha[t][.] among the B cached ones (those retained at step t - 1 plus the L tokens that just left
+ * the recent window; [0, B) at step 1; ties: lower position).  The L newest tokens are kept by the
+ * protocol and are not listed.
+ *   alpha_out: dev fp32 [M][T] (row t - 1 = step t); kept_out: dev int32 [M][B - L], ascending.
+ * B <= 8192 (FKV_ERR_CAPACITY beyond); M = 0 does nothing.  fkv_golden_select is the last step alone,
+ * from given future scores.
+ */
+int fkv_golden_steps(int32_t T, int32_t B, int32_t L);
+int fkv_golden_eviction(const float *attn, int32_t g, int32_t T, int32_t B, int32_t L, float *alpha_out,
+                        int32_t *kept_out, void *stream);
+int fkv_golden_select(const float *alpha, int32_t T, int32_t B, int32_t L, int32_t M, int32_t *kept_out, void *stream);
+
 /* Text of the last CUDA error seen by this library on this thread ("" if none). */
 const char *fkv_last_cuda_error(void);
 

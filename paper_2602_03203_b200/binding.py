@@ -26,7 +26,7 @@ EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", 
            "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
            "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
            "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing",
-           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled", "fkv_update_features", "fkv_evict_by_feature"]
+           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled", "fkv_update_features", "fkv_evict_by_feature", "fkv_golden_steps", "fkv_golden_eviction", "fkv_golden_select"]
 
 
 class FkvConfig(ctypes.Structure):
@@ -276,6 +276,28 @@ def decode_attn_dense_noalloc(q, k, v, group_size, out=None, scale=0.0):
                                                _ptr(out, torch.bfloat16), _stream())
     _check(code, "fkv_decode_attn_dense_noalloc")
     return out
+
+
+def golden_eviction(attn, B, L):
+    """Golden Eviction labels of one attention group: attn [g][T][T] fp32 on the device.
+    Returns (alpha [M][T], kept [M][B - L])."""
+    g, T, _ = attn.shape
+    M = lib().fkv_golden_steps(T, int(B), int(L))
+    if M < 0:
+        raise FkvError(M, "fkv_golden_steps")
+    alpha = torch.empty((M, T), dtype=torch.float32, device="cuda")
+    kept = torch.empty((M, B - L), dtype=torch.int32, device="cuda")
+    _check(lib().fkv_golden_eviction(_ptr(attn, torch.float32), g, T, int(B), int(L), _ptr(alpha, torch.float32),
+                                     _ptr(kept, torch.int32), _stream()), "fkv_golden_eviction")
+    return alpha, kept
+
+
+def golden_select(alpha, B, L):
+    M, T = alpha.shape
+    kept = torch.empty((M, B - L), dtype=torch.int32, device="cuda")
+    _check(lib().fkv_golden_select(_ptr(alpha, torch.float32), T, int(B), int(L), M, _ptr(kept, torch.int32), _stream()),
+           "fkv_golden_select")
+    return kept
 
 
 def pages_for(w, num_layers=None, extra_tokens=256) -> int:

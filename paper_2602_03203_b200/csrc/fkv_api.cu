@@ -18,6 +18,7 @@
 #include "fkv_compact.cuh"
 #include "fkv_dev.cuh"
 #include "fkv_features.cuh"
+#include "fkv_golden.cuh"
 #include "fkv_score.cuh"
 #include "fkv_select.cuh"
 
@@ -744,6 +745,47 @@ int fkv_launch_count(const fkv_cache *c, uint64_t *launches) {
   if (!c || !launches) return FKV_ERR_INVALID_ARG;
   *launches = c->launches;
   return FKV_OK;
+}
+
+static int golden_select_launch(const float *alpha, int T, int B, int L, int M, int32_t *kept, cudaStream_t st) {
+  int P = 1;
+  while (P < B) P <<= 1;
+  const size_t smem = (size_t)P * 8 + (size_t)B * 8;
+  if (B > 8192 || smem > kMaxSmem - 1024) return FKV_ERR_CAPACITY;
+  static size_t attr_bytes = 0;
+  if (smem > attr_bytes) {
+    FKV_CUDA(cudaFuncSetAttribute(k_golden_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_bytes = smem;
+  }
+  k_golden_select<<<1, 1024, smem, st>>>(alpha, T, B, L, M, P, kept);
+  FKV_CUDA(cudaGetLastError());
+  return FKV_OK;
+}
+
+int fkv_golden_steps(int32_t T, int32_t B, int32_t L) {
+  if (T < 1 || B < 2 || L < 1 || L >= B) return FKV_ERR_INVALID_ARG;
+  const int M = (T - B + L - 1) / L - 1;
+  return M < 0 ? 0 : M;
+}
+
+int fkv_golden_select(const float *alpha, int32_t T, int32_t B, int32_t L, int32_t M, int32_t *kept_out, void *stream) {
+  if (!alpha || !kept_out || M < 1 || fkv_golden_steps(T, B, L) < M) return FKV_ERR_INVALID_ARG;
+  return golden_select_launch(alpha, T, B, L, M, kept_out, (cudaStream_t)stream);
+}
+
+int fkv_golden_eviction(const float *attn, int32_t g, int32_t T, int32_t B, int32_t L, float *alpha_out,
+                        int32_t *kept_out, void *stream) {
+  if (!attn || !alpha_out || !kept_out || g < 1) return FKV_ERR_INVALID_ARG;
+  const int M = fkv_golden_steps(T, B, L);
+  if (M < 0) return M;
+  if (M == 0) return FKV_OK;
+  if (B > 8192) return FKV_ERR_CAPACITY;
+  cudaStream_t st = (cudaStream_t)stream;
+  k_golden_pool<<<dim3((T + 255) / 256, M), 256, 0, st>>>(attn, g, T, B, L, alpha_out);
+  FKV_CUDA(cudaGetLastError());
+  k_golden_suffix_max<<<(T + 255) / 256, 256, 0, st>>>(alpha_out, T, M);
+  FKV_CUDA(cudaGetLastError());
+  return golden_select_launch(alpha_out, T, B, L, M, kept_out, st);
 }
 
 const char *fkv_last_cuda_error(void) { return g_cuda_error.c_str(); }
