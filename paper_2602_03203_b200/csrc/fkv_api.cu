@@ -258,8 +258,8 @@ int launch_attend_t(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cud
 }
 
 int attend_dispatch(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cudaStream_t st) {
-  return c->cfg.head_dim == 128 ? launch_attend_t<128, 6, 12>(c, a, splits, pdl, st)
-                                : launch_attend_t<64, 8, 24>(c, a, splits, pdl, st);
+  return c->cfg.head_dim == 128 ? launch_attend_t<128, 4, 8>(c, a, splits, pdl, st)
+                                : launch_attend_t<64, 4, 16>(c, a, splits, pdl, st);
 }
 
 // Attention over `layer`, with the new pair of every participating sequence appended first when k_new is given.
