@@ -34,6 +34,23 @@ constexpr size_t kMaxSmem = 227 * 1024;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// The dynamic shared-memory opt-in is a per-device attribute of a kernel: remember, per kernel and per
+// device, the largest size already granted, and ask again only for more.
+struct SmemOptIn {
+  size_t granted[64] = {};
+  template <class Kernel>
+  cudaError_t ensure(Kernel kernel, size_t bytes) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    size_t &g = granted[dev & 63];
+    if (bytes <= g) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) g = bytes;
+    return e;
+  }
+};
+
 struct Layout {
   size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, hist_q, hist_ml, hist_n, hist_cnt, total;
   int cap, max_pages, num_pages, page_bytes, F, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
@@ -154,11 +171,8 @@ int launch_score(fkv_cache *c, float *out, int seg_base, int tiles_bound, cudaSt
   const int spw = score_slots_per_warp(c);
   if (spw == 0) return FKV_ERR_INVALID_ARG;
   const size_t smem = ScoreSmem::bytes(c->lay.page_bytes, c->lay.F, kScorePPS, spw);
-  static bool attr_done = false;
-  if (!attr_done) {
-    FKV_CUDA(cudaFuncSetAttribute(k_score<D, kScorePPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
-    attr_done = true;
-  }
+  static SmemOptIn opt_in;
+  FKV_CUDA(opt_in.ensure(k_score<D, kScorePPS>, kMaxSmem));
   const int grid = std::max(1, std::min(c->sm_count, tiles_bound));
   k_score<D, kScorePPS><<<grid, (kScorePPS + 1) * 32, smem, st>>>(c->ctx, out, seg_base, spw);
   FKV_LAUNCHED(c);
@@ -193,11 +207,8 @@ void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float
 template <int D>
 int launch_features_t(fkv_cache *c, int max_old, int nwork_bound, float scale_log2, cudaStream_t st) {
   const size_t smem = FeatSmem::bytes(D, c->lay.F, c->cfg.feature_window);
-  static size_t attr_bytes = 0;   // largest opt-in made so far
-  if (smem > attr_bytes) {
-    FKV_CUDA(cudaFuncSetAttribute(k_features<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_bytes = smem;
-  }
+  static SmemOptIn opt_in;
+  FKV_CUDA(opt_in.ensure(k_features<D>, smem));
   dim3 grid(((max_old + kPage - 1) / kPage + kFeatPages - 1) / kFeatPages, nwork_bound);
   if (grid.x == 0 || grid.y == 0) return FKV_OK;
   k_features<D><<<grid, 256, smem, st>>>(c->ctx, scale_log2);
@@ -752,11 +763,8 @@ static int golden_select_launch(const float *alpha, int T, int B, int L, int M, 
   while (P < B) P <<= 1;
   const size_t smem = (size_t)P * 8 + (size_t)B * 8;
   if (B > 8192 || smem > kMaxSmem - 1024) return FKV_ERR_CAPACITY;
-  static size_t attr_bytes = 0;
-  if (smem > attr_bytes) {
-    FKV_CUDA(cudaFuncSetAttribute(k_golden_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_bytes = smem;
-  }
+  static SmemOptIn opt_in;
+  FKV_CUDA(opt_in.ensure(k_golden_select, smem));
   k_golden_select<<<1, 1024, smem, st>>>(alpha, T, B, L, M, P, kept);
   FKV_CUDA(cudaGetLastError());
   return FKV_OK;
