@@ -211,6 +211,15 @@ int fkv_append_decode_attn(fkv_cache *c, int layer, const void *k, const void *v
  * step is (the next work on the stream is ordered after all of it).  For
  * engines that have all layers' tensors at hand, and for benchmarks of the
  * attention side alone.
+ *
+ * Stream capture: fkv_append_decode_attn and fkv_decode_step only enqueue
+ * kernels, so they may be recorded into a CUDA graph.  Every replay appends one
+ * more pair per sequence from the recorded k / v / q buffers: the kernel reads
+ * the lengths on the device, divides a segment's pages over the recorded number
+ * of splits whatever its length has become, and skips an append past
+ * max_tokens_per_head (FKV_DEV_CAPACITY).  The host's copy of the lengths does
+ * not see replays: call fkv_sync_lengths after the last replay and before any
+ * other call of this library.
  */
 int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *pos, const void *q, void *out,
                     float scale, void *stream);

@@ -49,7 +49,7 @@ struct AttendSmem {
   // ring | slot barriers (512 B) | received slices [kMaxSplits * per] (<= 8 * 128 + 16 floats) | received (m, l)
   static constexpr size_t kBars = 512, kRecvO = (8 * 128 + 4 * kMaxSplits) * 4, kRecvML = kMaxSplits * 8 * 2 * 4;
   static __host__ __device__ size_t ring(int D, int ncw, int slots) {
-    const size_t r = (size_t)slots * (4 * D * kPage), merge = (size_t)ncw * 8 * (D + 2) * 4;
+    const size_t r = (size_t)slots * (4 * D * kPage), merge = (size_t)ncw * 8 * (D + 4) * 4;
     return ((r > merge ? r : merge) + 127) & ~(size_t)127;
   }
   static __host__ __device__ size_t bytes(int D, int ncw, int slots) {
@@ -62,13 +62,15 @@ struct AttendArgs {
   const __nv_bfloat16 *q;   // [batch][Hkv * g][D]
   __nv_bfloat16 *out;       // same
   float scale_log2;         // softmax scale times log2(e)
-  int pps;                  // pages per split (>= 1); ceil(pages / pps) <= gridDim.x for every segment
+  int pps;                  // pages per split (>= 1) as the host sees the lengths; the kernel raises it where a segment is longer
   int append;               // 1: append k_new / v_new at slot n first (and record the query when the cache keeps a history)
   const uint8_t *k_new, *v_new;  // [batch][Hkv][D] bf16
   const int32_t *pos_new;   // [batch] or null (last position + 1)
   unsigned long long seq_mask;   // sequences that append (0 = all)
 };
 
+// The CTA-wide barrier, for the place where the producer warp and the consumer warps meet from different branches.
+__device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 0;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 // All threads of all CTAs of the cluster: writes made before (also into other CTAs' shared memory) are visible after.
 __device__ __forceinline__ void cluster_sync_all() {
@@ -80,8 +82,9 @@ __device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void dsmem_st(uint32_t addr, float v) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+__device__ __forceinline__ void dsmem_st4(uint32_t addr, float4 v) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+               : "memory");
 }
 __device__ __forceinline__ void dsmem_st2(uint32_t addr, float x, float y) {
   asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(x), "f"(y) : "memory");
@@ -94,20 +97,36 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
   constexpr int NCH = D / 8;   // 16-byte chunks per K (or V) row
   constexpr int PAGE_KV = 4 * D * kPage;
   static_assert(2 * NCH <= 32, "one chunk of the new row per lane");
-  static_assert(SLOTS <= 32 && 2 * SLOTS * 8 <= (int)AttendSmem::kBars, "one lane of the producer per slot");
+  static_assert(SLOTS <= 32 && 2 * SLOTS * 8 <= (int)AttendSmem::kBars, "the first SLOTS pages are issued one per lane");
   // A slot must always be consumed by the same warp: its barriers carry one parity bit, so a warp
   // waiting for the slot's next page may not run ahead of another warp's wait for the previous one.
   static_assert(SLOTS % NCW == 0, "slot s belongs to consumer warp s % NCW");
+  static_assert(32 % NCW == 0, "a group of NCW pages never straddles two 32-entry blocks of page ids");
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
   const int y = blockIdx.y, seq = y / c.Hkv, head = y % c.Hkv, G = c.G;
   const int S = gridDim.x, rank = blockIdx.x;   // the cluster is the grid's x extent
   const int seg = seg_of(c, a.layer, seq, head);
+  // The producer warp asks for its first page-table entries before the length is known, at the place the host's
+  // pages-per-split figure puts them (entries past the segment's pages are never used), so that the two reads
+  // overlap instead of following one another.
+  int *ptrow = c.pt + (size_t)seg * c.max_pages;
+  int ptv = 0, ptn = 0;
+  if (warp == NCW) {
+    const int e = rank * a.pps + lane;
+    if (e < c.max_pages) ptv = ptrow[e];
+    if (e + 32 < c.max_pages) ptn = ptrow[e + 32];
+  }
   const int n_old = c.len[a.layer * c.batch + seq];
-  const bool app = a.append && (!a.seq_mask || ((a.seq_mask >> seq) & 1ull));
+  // The host refuses an append past the capacity; a replayed launch (CUDA graph) is checked here instead.
+  const bool want = a.append && (!a.seq_mask || ((a.seq_mask >> seq) & 1ull));
+  const bool app = want && n_old < c.cap;
+  if (want && !app && tid == 0 && rank == 0) set_status(c, kDevCapacity);
   const int n = n_old + (app ? 1 : 0);
   const int npages = (n + kPage - 1) / kPage;
-  const int pg0 = rank * a.pps, pg1 = min(npages, pg0 + a.pps);
+  // Pages per split: the host's figure, or more when the segment has outgrown it since the launch was recorded.
+  const int pps = max(a.pps, (npages + S - 1) >> (31 - __clz(S)));   // S is a power of two
+  const int pg0 = rank * pps, pg1 = min(npages, pg0 + pps);
   const bool active = pg0 < pg1;
   const int npg = active ? pg1 - pg0 : 0;               // pages of this CTA
   const bool tail = app && active && pg1 == npages;     // this CTA's range holds the new pair
@@ -123,37 +142,48 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + ring_bytes);                      // full[SLOTS], empty[SLOTS]
   float *recv_o = reinterpret_cast<float *>(smem + ring_bytes + AttendSmem::kBars);      // [S][per]: my slice of every partial
   float *recv_ml = reinterpret_cast<float *>(smem + ring_bytes + AttendSmem::kBars + AttendSmem::kRecvO);  // [S][8][2]
-  if (tid == 0) {
-    griddep_launch();   // nothing here depends on, or is needed by, the next launch of a decode step
-    for (int s = 0; s < 2 * SLOTS; ++s) mbar_init(smem_u32(&bars[s]), 1);
-    fence_barrier_init();
-  }
-  __syncthreads();   // every thread has read the length by now (the length bump at the end relies on it)
-
   const int gid = lane >> 2, tig = lane & 3;
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // queries 2 tig and 2 tig + 1
   float o[MT][4];
 #pragma unroll
   for (int i = 0; i < MT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
 
-  if (active && warp == NCW) {
-    // ---------------- producer: lane l < SLOTS owns slot l and moves pages l, l + SLOTS, ... into it, in order
-    // (a slot's barriers carry one parity bit, so its pages must be issued one phase at a time) ----------------
-    int *ptrow = c.pt + (size_t)seg * c.max_pages;
-    auto issue = [&](int i, int pid) {   // page i of the CTA into slot i % SLOTS
-      const uint32_t full = smem_u32(&bars[i % SLOTS]);
-      if (fresh && pg0 + i == npages - 1) {
-        mbar_arrive(full);               // a brand-new page: the consumer builds it
-      } else {
-        mbar_arrive_expect_tx(full, PAGE_KV);
-        bulk_g2s(smem_u32(smem + (size_t)(i % SLOTS) * PAGE_KV), c.pool + (size_t)pid * c.page_bytes, PAGE_KV, full);
-      }
-    };
-    const bool owner = lane < SLOTS;
-    int pid = owner && lane < npg ? ptrow[pg0 + lane] : 0;
-    int nxt = owner && lane + SLOTS < npg ? ptrow[pg0 + lane + SLOTS] : 0;
-    if (owner && lane < npg) issue(lane, pid);   // the ring is empty: no wait
+  // The cache is far larger than L2 and every page is read once per token: mark the pages evict-first so that
+  // the small state every launch starts from (lengths, page tables) tends to stay in L2.
+  const uint64_t stream_policy = l2_policy_evict_first();
+  auto issue = [&](int i, int pid) {   // page i of the CTA into slot i % SLOTS
+    const uint32_t full = smem_u32(&bars[i % SLOTS]);
+    if (fresh && pg0 + i == npages - 1) {
+      mbar_arrive(full);               // a brand-new page: the consumer builds it
+    } else {
+      mbar_arrive_expect_tx(full, PAGE_KV);
+      bulk_g2s_hint(smem_u32(smem + (size_t)(i % SLOTS) * PAGE_KV), c.pool + (size_t)pid * c.page_bytes, PAGE_KV, full,
+                    stream_policy);
+    }
+  };
+
+  if (warp == NCW) {
+    // ---------------- producer: page i of the CTA goes to slot i % SLOTS; pages are issued in page order, so a
+    // slot's barriers (one parity bit each) see exactly one phase at a time.  The warp sets the barriers up itself
+    // and fills the empty ring before it meets the consumers at the CTA barrier. ----------------
+    if (lane == 0) {
+      for (int s = 0; s < 2 * SLOTS; ++s) mbar_init(smem_u32(&bars[s]), 1);
+      fence_barrier_init();
+    }
     __syncwarp();
+    // ptv / ptn: page ids of the CTA's pages [0, 32) and [32, 64), one per lane.
+    if (active && pps != a.pps) {   // the early read looked in the wrong place
+      ptv = lane < npg ? ptrow[pg0 + lane] : 0;
+      ptn = 32 + lane < npg ? ptrow[pg0 + 32 + lane] : 0;
+    }
+    if (lane < SLOTS && lane < npg) issue(lane, ptv);         // the ring is empty: no wait
+    cta_sync();
+  } else {
+    if (tid == 0) griddep_launch();   // nothing here depends on, or is needed by, the next launch of a decode step
+    cta_sync();                       // the barriers are set up
+  }
+
+  if (active && warp == NCW) {
     if (tail) {
       // The new pair goes to slot n_old of the page record (and, below, into the consumer's copy of the page).
       int npid = -1;
@@ -185,14 +215,25 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
       }
       __syncwarp();
     }
-    // The pages that did not fit the empty ring: each waits for the previous page of its slot to be consumed.
-    if (owner)
-      for (int i = lane + SLOTS; i < npg; i += SLOTS) {
-        pid = nxt;
-        if (i + SLOTS < npg) nxt = ptrow[pg0 + i + SLOTS];
-        if (!mbar_wait(smem_u32(&bars[SLOTS + lane]), ((i / SLOTS) & 1) ^ 1)) { set_status(c, kDevWaitTimeout); break; }
-        issue(i, pid);
+    // The pages that did not fit the empty ring, in page order and NCW at a time (one page of every consumer warp:
+    // their slots come free together).  The whole warp waits, converged, for the previous pages of the group's
+    // slots to be consumed; then lanes 0 .. NCW-1 issue one copy each.
+    for (int i = SLOTS; i < npg; i += NCW) {
+      if ((i & 31) == 0) {
+        ptv = ptn;
+        ptn = i + 32 + lane < npg ? ptrow[pg0 + i + 32 + lane] : 0;
       }
+      const int pid = __shfl_sync(0xffffffffu, ptv, (i + lane) & 31);
+      bool ok = true;
+#pragma unroll
+      for (int j = 0; j < NCW; ++j)
+        if (i + j < npg) ok = ok && mbar_wait(smem_u32(&bars[SLOTS + (i + j) % SLOTS]), (((i + j) / SLOTS) & 1) ^ 1);
+      if (!__all_sync(0xffffffffu, ok)) {
+        if (lane == 0) set_status(c, kDevWaitTimeout);
+        break;
+      }
+      if (lane < NCW && i + lane < npg) issue(i + lane, pid);
+    }
   } else if (active) {
     // ---------------- consumers: warp w takes pages w, w + NCW, ... of this CTA ----------------
     // Q^T as B fragments (channels x queries): column gid = query head gid of the group (zero beyond g).
@@ -280,10 +321,11 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
   }
   __syncthreads();  // every issued copy has landed and been consumed: the ring can be reused
 
-  // ---- merge the consumer warps of this CTA: smem [NCW][8 queries][D + 2] ----
+  // ---- merge the consumer warps of this CTA: smem [NCW][8 queries][D + 4] (rows 16-byte aligned) ----
+  constexpr int MGS = D + 4;
   float *mg = reinterpret_cast<float *>(smem);
   if (active && warp < NCW) {
-    float *r0 = mg + ((size_t)warp * 8 + 2 * tig) * (D + 2), *r1 = r0 + (D + 2);
+    float *r0 = mg + ((size_t)warp * 8 + 2 * tig) * MGS, *r1 = r0 + MGS;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       r0[mt * 16 + gid] = o[mt][0]; r1[mt * 16 + gid] = o[mt][1];
@@ -293,57 +335,96 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
   }
   __syncthreads();
 
-  // ---- push: element e of the merged partial goes to the CTA that owns e / per (its slot `rank`) ----
-  const int per = (G * D + S - 1) / S;   // output elements per owner
+  // ---- push: elements [o * per, (o + 1) * per) of the merged partial go to CTA o of the cluster (its slot
+  // `rank`), four channels per store; the producer warp sends the (m, l) of every query row to every CTA ----
+  const int per = G * D / S;   // output elements per owner: S is a power of two <= 16 and 64 divides G * D
   const uint32_t recv_o_s = smem_u32(recv_o), recv_ml_s = smem_u32(recv_ml);
-  for (int e = tid; e < G * D; e += blockDim.x) {
-    const int r = e / D, ch = e - r * D;
-    float acc = 0.f;
-    if (active) {
-      float M = -INFINITY;
+  if (warp < NCW) {
+    for (int e = tid * 4; e < G * D; e += NCW * 32 * 4) {
+      const int r = e / D, ch = e - r * D;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (active) {
+        float mw[NCW], M = -INFINITY;
 #pragma unroll
-      for (int w = 0; w < NCW; ++w) M = fmaxf(M, mg[((size_t)w * 8 + r) * (D + 2) + D]);
+        for (int w = 0; w < NCW; ++w) {
+          mw[w] = mg[((size_t)w * 8 + r) * MGS + D];
+          M = fmaxf(M, mw[w]);
+        }
 #pragma unroll
-      for (int w = 0; w < NCW; ++w) {
-        const float *rw = mg + ((size_t)w * 8 + r) * (D + 2);
-        acc += (rw[D] == -INFINITY ? 0.f : exp2f(rw[D] - M)) * rw[ch];
+        for (int w = 0; w < NCW; ++w) {
+          const float f = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);
+          const float4 x = *reinterpret_cast<const float4 *>(mg + ((size_t)w * 8 + r) * MGS + ch);
+          acc.x = fmaf(f, x.x, acc.x); acc.y = fmaf(f, x.y, acc.y);
+          acc.z = fmaf(f, x.z, acc.z); acc.w = fmaf(f, x.w, acc.w);
+        }
       }
+      const int owner = e / per;
+      dsmem_st4(dsmem_addr(recv_o_s + (uint32_t)(rank * per + (e - owner * per)) * 4u, owner), acc);
     }
-    const int owner = e / per;
-    dsmem_st(dsmem_addr(recv_o_s + (uint32_t)(rank * per + (e - owner * per)) * 4u, owner), acc);
-  }
-  for (int e = tid; e < S * G; e += blockDim.x) {   // (m, l) of every query row, to every CTA
-    const int owner = e / G, r = e - owner * G;
-    float M = -INFINITY, l = 0.f;
-    if (active) {
+  } else {
+    for (int e = lane; e < S * G; e += 32) {
+      const int owner = e / G, r = e - owner * G;
+      float M = -INFINITY, l = 0.f;
+      if (active) {
 #pragma unroll
-      for (int w = 0; w < NCW; ++w) M = fmaxf(M, mg[((size_t)w * 8 + r) * (D + 2) + D]);
+        for (int w = 0; w < NCW; ++w) M = fmaxf(M, mg[((size_t)w * 8 + r) * MGS + D]);
 #pragma unroll
-      for (int w = 0; w < NCW; ++w) {
-        const float *rw = mg + ((size_t)w * 8 + r) * (D + 2);
-        l += (rw[D] == -INFINITY ? 0.f : exp2f(rw[D] - M)) * rw[D + 1];
+        for (int w = 0; w < NCW; ++w) {
+          const float *rw = mg + ((size_t)w * 8 + r) * MGS;
+          l += (rw[D] == -INFINITY ? 0.f : exp2f(rw[D] - M)) * rw[D + 1];
+        }
       }
+      dsmem_st2(dsmem_addr(recv_ml_s + (uint32_t)(rank * 8 + r) * 8u, owner), M, l);
     }
-    dsmem_st2(dsmem_addr(recv_ml_s + (uint32_t)(rank * 8 + r) * 8u, owner), M, l);
   }
   cluster_sync_all();
 
-  // ---- reduce the slice this CTA owns over the S partials and write it ----
-  for (int e = tid; e < per; e += blockDim.x) {
-    const int ge = rank * per + e;
-    if (ge >= G * D) break;
-    const int r = ge / D;
-    float M = -INFINITY;
-    for (int s = 0; s < S; ++s) M = fmaxf(M, recv_ml[(s * 8 + r) * 2]);
-    float acc = 0.f, L = 0.f;
-    for (int s = 0; s < S; ++s) {
-      const float ms = recv_ml[(s * 8 + r) * 2];
-      const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
-      L = fmaf(f, recv_ml[(s * 8 + r) * 2 + 1], L);
-      acc = fmaf(f, recv_o[s * per + e], acc);
+  // ---- reduce the slice this CTA owns, [rank * per, (rank + 1) * per), over the S partials and write it: one
+  // warp per query row of the slice; lane s holds the statistics of partial s; the lanes form 4 groups that each
+  // sum every fourth partial for 8 x 4 channels, and the groups are added with shuffles ----
+  const int lo = rank * per, hi = lo + per;
+  for (int r = lo / D + warp; r * D < hi; r += NCW + 1) {
+    const int e0 = max(lo, r * D), e1 = min(hi, (r + 1) * D);
+    const float ms = lane < S ? recv_ml[(lane * 8 + r) * 2] : -INFINITY;
+    const float ls = lane < S ? recv_ml[(lane * 8 + r) * 2 + 1] : 0.f;
+    float M = ms;
+#pragma unroll
+    for (int sh = 16; sh >= 1; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+    const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
+    float L = f * ls;
+#pragma unroll
+    for (int sh = 16; sh >= 1; sh >>= 1) L += __shfl_xor_sync(0xffffffffu, L, sh);
+    const float inv = L > 0.f ? 1.f / L : 0.f;   // an empty sequence gives zeros
+    const int grp = lane >> 3, l8 = lane & 7;
+    for (int base = e0; base < e1; base += 32) {
+      const int e = base + l8 * 4;
+      const bool valid = e < e1;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int k = 0; k < kMaxSplits / 4; ++k) {
+        const int sp = grp + 4 * k;
+        const float fs = __shfl_sync(0xffffffffu, f, sp);
+        if (sp < S && valid) {
+          const float4 x = *reinterpret_cast<const float4 *>(recv_o + sp * per + (e - lo));
+          acc.x = fmaf(fs, x.x, acc.x); acc.y = fmaf(fs, x.y, acc.y);
+          acc.z = fmaf(fs, x.z, acc.z); acc.w = fmaf(fs, x.w, acc.w);
+        }
+      }
+#pragma unroll
+      for (int sh = 8; sh <= 16; sh <<= 1) {
+        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, sh); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, sh);
+        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, sh); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, sh);
+      }
+      if (grp == 0 && valid) {
+        const __nv_bfloat162 p0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+        const __nv_bfloat162 p1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t *>(&p0);
+        pk.y = *reinterpret_cast<const uint32_t *>(&p1);
+        *reinterpret_cast<uint2 *>(a.out + qrow0 * D + e) = pk;
+      }
     }
-    a.out[qrow0 * D + ge] = __float2bfloat16(L > 0.f ? acc / L : 0.f);   // an empty sequence gives zeros
-    if (rec && ge - r * D == 0) reinterpret_cast<float2 *>(c.hist_ml)[hrow + r] = make_float2(M, L);
+    if (rec && e0 == r * D && lane == 0) reinterpret_cast<float2 *>(c.hist_ml)[hrow + r] = make_float2(M, L);
   }
   if (rec && rank == 0)   // the queries themselves: G rows of D bf16
     for (int i = tid; i < G * D / 8; i += blockDim.x)
