@@ -52,8 +52,8 @@ struct SmemOptIn {
 };
 
 struct Layout {
-  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, hist_q, hist_ml, hist_n, hist_cnt, total;
-  int cap, max_pages, num_pages, page_bytes, F, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
+  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, att_part, att_tickets, hist_q, hist_ml, hist_n, hist_cnt, total;
+  int cap, max_pages, num_pages, page_bytes, F, att_smax, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
 };
 
 bool valid_config(const fkv_config *c) {
@@ -104,6 +104,10 @@ Layout make_layout(const fkv_config &c) {
   L.work = take(nseg * 4);
   L.tile1 = take((nseg + 1) * 4);
   L.seq_tickets = take((size_t)c.num_layers * c.max_batch * 4);
+  // Split-K attention: up to att_smax splits per segment (enough for a few CTAs per SM at this batch size).
+  L.att_smax = std::max(1, std::min(kMaxSplits, 512 / (c.max_batch * c.num_kv_heads)));
+  L.att_part = take(nseg * L.att_smax * c.group_size * (D + 4) * 4);
+  L.att_tickets = take(nseg * 4);
   const size_t ls = (size_t)c.num_layers * c.max_batch, W = (size_t)c.feature_window, Hq = (size_t)c.num_kv_heads * c.group_size;
   L.hist_q = take(ls * W * Hq * D * 2);
   L.hist_ml = take(ls * W * Hq * 8);
@@ -134,7 +138,6 @@ struct fkv_cache {
   uint64_t launches = 0;
   int sm_count = 148;
   float feature_scale = 0.f;  // softmax scale of the recorded queries (the last decode call's)
-  int max_cluster = 0;  // largest attention cluster this device places (found at the first launch)
   bool timing = false, timed = false;
   cudaEvent_t ev[7] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};  // [6]: after the plan
 };
@@ -230,39 +233,24 @@ int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, 
   return FKV_OK;
 }
 
-// One launch of the attention kernel: the `splits` CTAs of a segment are one cluster.  a == nullptr does the
-// once-per-handle set-up instead.  pdl: the launch may run alongside the one before it on the stream.
+// One launch of the attention kernel: `splits` CTAs per segment.  pdl: the launch may run alongside the one
+// before it on the stream.
 template <int D, int NCW, int SLOTS>
 int launch_attend_t(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cudaStream_t st) {
   const size_t smem = AttendSmem::bytes(D, NCW, SLOTS);
   auto kern = k_attend<D, NCW, SLOTS>;
+  static SmemOptIn opt_in;
+  FKV_CUDA(opt_in.ensure(kern, smem));
   cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(splits, c->cfg.max_batch * c->cfg.num_kv_heads);
   cfg.blockDim = dim3((NCW + 1) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute at[2];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  if (!a) {
-    // Opt in to the shared memory and to clusters of 16, and find the largest cluster (16, else 8) this
-    // device can actually place.
-    FKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    FKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-    cfg.gridDim = dim3(16, 1);
-    at[0].val.clusterDim.x = 16;
-    cfg.numAttrs = 1;
-    int nclusters = 0;
-    const bool ok16 = cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg) == cudaSuccess && nclusters > 0;
-    (void)cudaGetLastError();
-    c->max_cluster = ok16 ? 16 : 8;
-    return FKV_OK;
-  }
-  cfg.gridDim = dim3(splits, c->cfg.max_batch * c->cfg.num_kv_heads);
-  at[0].val.clusterDim.x = splits;
-  cfg.numAttrs = pdl ? 2 : 1;
+  cfg.numAttrs = pdl ? 1 : 0;
   FKV_CUDA(cudaLaunchKernelEx(&cfg, kern, c->ctx, *a));
   ++c->launches;
   return FKV_OK;
@@ -283,16 +271,11 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
     const int n = c->h_len[(size_t)layer * batch + s] + ((app && (!seq_mask || ((seq_mask >> s) & 1ull))) ? 1 : 0);
     maxpages = std::max(maxpages, (n + kPage - 1) / kPage);
   }
-  if (c->max_cluster == 0) {
-    const int rc = attend_dispatch(c, nullptr, 0, false, st);
-    if (rc) return rc;
-  }
-  // Splits per segment: a power of two, about two CTAs per SM in total, at least kAttendMinPages pages each.
-  const int nseg = batch * Hkv, cap = std::min(c->max_cluster, kMaxSplits);
-  int splits = 1;
-  while (splits * 2 <= cap && splits * 2 * nseg <= 2 * c->sm_count &&
-         (maxpages + splits * 2 - 1) / (splits * 2) >= kAttendMinPages)
-    splits *= 2;
+  // Splits per segment: CTAs for about three quarters of the SMs per launch (consecutive launches of a decode
+  // step share the SMs, three CTAs fit on one), at least kAttendMinPages pages each.
+  const int nseg = batch * Hkv;
+  int splits = std::min(c->lay.att_smax, std::max(1, (c->sm_count * 3 / 4 + nseg / 2) / nseg));
+  splits = std::max(1, std::min(splits, maxpages / kAttendMinPages));
   const int pps = std::max(1, (maxpages + splits - 1) / splits);
   if (scale == 0.f) scale = 1.f / sqrtf((float)D);
   if (app) c->feature_scale = scale;
@@ -341,6 +324,7 @@ int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, voi
   x.scores = (float *)(ws + L.scores); x.idx = (int *)(ws + L.idx); x.plan = (SegPlan *)(ws + L.plan);
   x.work = (int *)(ws + L.work); x.tile1_start = (int *)(ws + L.tile1);
   x.seq_tickets = (int *)(ws + L.seq_tickets);
+  x.att_part = (float *)(ws + L.att_part); x.att_tickets = (int *)(ws + L.att_tickets); x.att_smax = L.att_smax;
   x.hist_w = cfg->feature_window; x.hist_q = ws + L.hist_q; x.hist_ml = (float *)(ws + L.hist_ml);
   x.hist_n = (int *)(ws + L.hist_n); x.hist_cnt = (int *)(ws + L.hist_cnt);
   c->h_len.assign((size_t)cfg->num_layers * cfg->max_batch, 0);

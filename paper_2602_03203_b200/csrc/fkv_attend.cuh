@@ -5,21 +5,23 @@
 //
 // Roofline: HBM, 4D bytes per retained pair per token.
 //
-// Shape: grid (splits, sequences x KV heads); the `splits` CTAs of a segment
-// form ONE thread-block cluster, each walking a contiguous range of pages.
+// Shape: grid (splits, sequences x KV heads); each of the `splits` CTAs of a
+// segment walks a contiguous range of its pages.
 //   - A producer warp copies the K|V part of each page record (one contiguous
 //     4D*16-byte block) into a ring of page slots with bulk async copies, one
-//     full/empty mbarrier pair per slot.
+//     full/empty mbarrier pair per slot.  Pages are issued in page order, NCW
+//     at a time, by a converged warp.
 //   - NCW consumer warps take pages round-robin, each on its own: keys sit on
 //     the M axis of the mma (S^T = K Q^T, 16 keys x 8 query columns, columns
 //     >= g zero), softmax is online in fp32 with exp2, the two 8 x 8 tiles of
 //     P^T are transposed in registers (movmatrix) into the B operand of
 //     O^T = V^T P^T, whose A operand comes from ldmatrix.trans on V.
-//   - The warps' (m, l, O) are merged in shared memory; every CTA then PUSHES
-//     its merged partial, slice by slice, into the shared memory of the CTA
-//     that owns that slice of the output (distributed shared memory), one
-//     cluster barrier follows, and every CTA reduces and writes its own slice.
-//     No partial ever goes to global memory and nobody spins.
+//   - The warps' (m, l, O) are merged in shared memory and the CTA's partial
+//     goes to a small global buffer (it never leaves L2); an arrival counter
+//     per segment tells the last CTA to finish, which merges the partials (one
+//     round trip to L2, every load in flight at once) and writes the output.
+//     A CTA that is not last exits as soon as its partial is out, so its
+//     shared memory is free for the next launch.
 //
 // The launch can also APPEND the token's new (k, v) pair first (Section 3.1:
 // the cache grows by one pair per generated token): the CTA whose page range
@@ -36,25 +38,23 @@
 // that has every layer's tensors at hand can therefore launch layer l with the
 // programmatic-dependent-launch attribute: its CTAs start as soon as layer
 // l-1's CTAs are all running and stream their pages while those still
-// compute (a CTA needs under half an SM, so consecutive launches are
-// co-resident).  Without the attribute the launch is ordered like any other.
+// compute (three CTAs fit on an SM, so consecutive launches are co-resident).
+// Without the attribute the launch is ordered like any other.
 #pragma once
 #include "fkv_dev.cuh"
 
 namespace fkv {
 
-constexpr int kMaxSplits = 16;   // CTAs per cluster = splits per segment
+constexpr int kMaxSplits = 32;   // splits per segment (one lane of the merging warp per split)
 
 struct AttendSmem {
-  // ring | slot barriers (512 B) | received slices [kMaxSplits * per] (<= 8 * 128 + 16 floats) | received (m, l)
-  static constexpr size_t kBars = 512, kRecvO = (8 * 128 + 4 * kMaxSplits) * 4, kRecvML = kMaxSplits * 8 * 2 * 4;
+  // ring | slot barriers (512 B)
+  static constexpr size_t kBars = 512;
   static __host__ __device__ size_t ring(int D, int ncw, int slots) {
     const size_t r = (size_t)slots * (4 * D * kPage), merge = (size_t)ncw * 8 * (D + 4) * 4;
     return ((r > merge ? r : merge) + 127) & ~(size_t)127;
   }
-  static __host__ __device__ size_t bytes(int D, int ncw, int slots) {
-    return ring(D, ncw, slots) + kBars + kRecvO + kRecvML;
-  }
+  static __host__ __device__ size_t bytes(int D, int ncw, int slots) { return ring(D, ncw, slots) + kBars; }
 };
 
 struct AttendArgs {
@@ -72,26 +72,101 @@ struct AttendArgs {
 // The CTA-wide barrier, for the place where the producer warp and the consumer warps meet from different branches.
 __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 0;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-// All threads of all CTAs of the cluster: writes made before (also into other CTAs' shared memory) are visible after.
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Address of this CTA's shared-memory location `local` in CTA `rank` of the cluster.
-__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void dsmem_st4(uint32_t addr, float4 v) {
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
-               : "memory");
-}
-__device__ __forceinline__ void dsmem_st2(uint32_t addr, float x, float y) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(x), "f"(y) : "memory");
+// The merge of a segment's split partials, run by the whole CTA that finished last.  part: [nact][G][D + 4] fp32
+// (O relative to the partial's own maximum, then m and l); out: G rows of D bf16; scratch: shared memory,
+// NW * 8 * D + 16 floats.  One round trip to L2 per pass: warp w asks for partials w, w + NW, ... (PASS of them
+// per pass, all query rows, four channels per lane) and, lane s, for the statistics of partial s, before it uses
+// any of them.  R = query rows handled (>= G), a compile-time bound that sizes the register arrays.
+template <int D, int NW, int R, int PASS>
+__device__ __forceinline__ void merge_partials(const float *part, int nact, int G, float *scratch, __nv_bfloat16 *out,
+                                               float2 *hist_ml) {
+  constexpr int PRS = D + 4;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
+  float *red = scratch;               // [NW][8][D]: one partial sum per warp
+  float *tot = red + NW * 8 * D;      // [8]: 1 / L of every query row
+  const bool mine = lane < D / 4;
+  float2 st[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+    st[r] = (r < G && lane < nact) ? __ldcg(reinterpret_cast<const float2 *>(part + ((size_t)lane * G + r) * PRS + D))
+                                   : make_float2(-INFINITY, 0.f);
+  float4 acc[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+  float Mr[R];
+  bool have_max = false;
+  for (int sp0 = warp; sp0 < nact; sp0 += NW * PASS) {
+    float4 x[PASS][R];
+#pragma unroll
+    for (int k = 0; k < PASS; ++k)
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const int sp = sp0 + k * NW;
+        x[k][r] = (mine && r < G && sp < nact)
+                      ? __ldcg(reinterpret_cast<const float4 *>(part + ((size_t)sp * G + r) * PRS + lane * 4))
+                      : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    if (!have_max) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        float M = st[r].x;
+#pragma unroll
+        for (int sh = 16; sh >= 1; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+        Mr[r] = M;
+      }
+      have_max = true;
+    }
+#pragma unroll
+    for (int k = 0; k < PASS; ++k)
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const int sp = sp0 + k * NW;
+        const float ms = __shfl_sync(0xffffffffu, st[r].x, sp & 31);
+        const float fs = (sp < nact && ms != -INFINITY) ? exp2f(ms - Mr[r]) : 0.f;
+        acc[r].x = fmaf(fs, x[k][r].x, acc[r].x); acc[r].y = fmaf(fs, x[k][r].y, acc[r].y);
+        acc[r].z = fmaf(fs, x[k][r].z, acc[r].z); acc[r].w = fmaf(fs, x[k][r].w, acc[r].w);
+      }
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+    if (r < G && mine) *reinterpret_cast<float4 *>(red + ((size_t)warp * 8 + r) * D + lane * 4) = acc[r];
+  if (warp == NW - 1) {   // the totals of every row: M, then L = sum_s exp2(m_s - M) l_s
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float M = st[r].x;
+#pragma unroll
+      for (int sh = 16; sh >= 1; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+      float L = st[r].x == -INFINITY ? 0.f : exp2f(st[r].x - M) * st[r].y;
+#pragma unroll
+      for (int sh = 16; sh >= 1; sh >>= 1) L += __shfl_xor_sync(0xffffffffu, L, sh);
+      if (lane == 0 && r < G) {
+        tot[r] = L > 0.f ? 1.f / L : 0.f;   // an empty sequence gives zeros
+        if (hist_ml) hist_ml[r] = make_float2(M, L);
+      }
+    }
+  }
+  __syncthreads();
+  // Sum over the warps, normalise, write: one thread per four channels of a query row.
+  for (int e = tid * 4; e < G * D; e += blockDim.x * 4) {
+    const int r = e / D, ch = e - r * D;
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float4 v = *reinterpret_cast<const float4 *>(red + ((size_t)w * 8 + r) * D + ch);
+      sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+    }
+    const float inv = tot[r];
+    const __nv_bfloat162 p0 = __floats2bfloat162_rn(sum.x * inv, sum.y * inv);
+    const __nv_bfloat162 p1 = __floats2bfloat162_rn(sum.z * inv, sum.w * inv);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t *>(&p0);
+    pk.y = *reinterpret_cast<const uint32_t *>(&p1);
+    *reinterpret_cast<uint2 *>(out + r * D + ch) = pk;
+  }
 }
 
 template <int D, int NCW, int SLOTS>
-__global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) {
+__global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx c, AttendArgs a) {
   constexpr int KSQ = D / 16;  // k-steps of K Q^T
   constexpr int MT = D / 16;   // m-tiles (16 channels) of O^T = V^T P^T
   constexpr int NCH = D / 8;   // 16-byte chunks per K (or V) row
@@ -105,7 +180,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
   const int y = blockIdx.y, seq = y / c.Hkv, head = y % c.Hkv, G = c.G;
-  const int S = gridDim.x, rank = blockIdx.x;   // the cluster is the grid's x extent
+  const int S = gridDim.x, rank = blockIdx.x;   // splits of the segment, and this CTA's
   const int seg = seg_of(c, a.layer, seq, head);
   // The producer warp asks for its first page-table entries before the length is known, at the place the host's
   // pages-per-split figure puts them (entries past the segment's pages are never used), so that the two reads
@@ -125,7 +200,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
   const int n = n_old + (app ? 1 : 0);
   const int npages = (n + kPage - 1) / kPage;
   // Pages per split: the host's figure, or more when the segment has outgrown it since the launch was recorded.
-  const int pps = max(a.pps, (npages + S - 1) >> (31 - __clz(S)));   // S is a power of two
+  const int pps = max(a.pps, (npages + S - 1) / S);
   const int pg0 = rank * pps, pg1 = min(npages, pg0 + pps);
   const bool active = pg0 < pg1;
   const int npg = active ? pg1 - pg0 : 0;               // pages of this CTA
@@ -140,8 +215,6 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
 
   const size_t ring_bytes = AttendSmem::ring(D, NCW, SLOTS);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + ring_bytes);                      // full[SLOTS], empty[SLOTS]
-  float *recv_o = reinterpret_cast<float *>(smem + ring_bytes + AttendSmem::kBars);      // [S][per]: my slice of every partial
-  float *recv_ml = reinterpret_cast<float *>(smem + ring_bytes + AttendSmem::kBars + AttendSmem::kRecvO);  // [S][8][2]
   const int gid = lane >> 2, tig = lane & 3;
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // queries 2 tig and 2 tig + 1
   float o[MT][4];
@@ -335,21 +408,22 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
   }
   __syncthreads();
 
-  // ---- push: elements [o * per, (o + 1) * per) of the merged partial go to CTA o of the cluster (its slot
-  // `rank`), four channels per store; the producer warp sends the (m, l) of every query row to every CTA ----
-  const int per = G * D / S;   // output elements per owner: S is a power of two <= 16 and 64 divides G * D
-  const uint32_t recv_o_s = smem_u32(recv_o), recv_ml_s = smem_u32(recv_ml);
-  if (warp < NCW) {
-    for (int e = tid * 4; e < G * D; e += NCW * 32 * 4) {
-      const int r = e / D, ch = e - r * D;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (active) {
+  // ---- this CTA's partial, relative to its own maximum, goes to global memory (it stays in L2): per query row
+  // D floats of O, then m and l ----
+  constexpr int PRS = D + 4;   // floats per row of a partial record
+  float *seg_part = c.att_part + (size_t)seg * c.att_smax * G * PRS;
+  if (active) {
+    float *part = seg_part + (size_t)rank * G * PRS;
+    if (warp < NCW) {
+      for (int e = tid * 4; e < G * D; e += NCW * 32 * 4) {
+        const int r = e / D, ch = e - r * D;
         float mw[NCW], M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < NCW; ++w) {
           mw[w] = mg[((size_t)w * 8 + r) * MGS + D];
           M = fmaxf(M, mw[w]);
         }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int w = 0; w < NCW; ++w) {
           const float f = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);
@@ -357,74 +431,39 @@ __global__ void __launch_bounds__((NCW + 1) * 32) k_attend(Ctx c, AttendArgs a) 
           acc.x = fmaf(f, x.x, acc.x); acc.y = fmaf(f, x.y, acc.y);
           acc.z = fmaf(f, x.z, acc.z); acc.w = fmaf(f, x.w, acc.w);
         }
+        __stcg(reinterpret_cast<float4 *>(part + r * PRS + ch), acc);
       }
-      const int owner = e / per;
-      dsmem_st4(dsmem_addr(recv_o_s + (uint32_t)(rank * per + (e - owner * per)) * 4u, owner), acc);
-    }
-  } else {
-    for (int e = lane; e < S * G; e += 32) {
-      const int owner = e / G, r = e - owner * G;
+    } else if (lane < G) {
+      const int r = lane;
       float M = -INFINITY, l = 0.f;
-      if (active) {
 #pragma unroll
-        for (int w = 0; w < NCW; ++w) M = fmaxf(M, mg[((size_t)w * 8 + r) * MGS + D]);
+      for (int w = 0; w < NCW; ++w) M = fmaxf(M, mg[((size_t)w * 8 + r) * MGS + D]);
 #pragma unroll
-        for (int w = 0; w < NCW; ++w) {
-          const float *rw = mg + ((size_t)w * 8 + r) * MGS;
-          l += (rw[D] == -INFINITY ? 0.f : exp2f(rw[D] - M)) * rw[D + 1];
-        }
+      for (int w = 0; w < NCW; ++w) {
+        const float *rw = mg + ((size_t)w * 8 + r) * MGS;
+        l += (rw[D] == -INFINITY ? 0.f : exp2f(rw[D] - M)) * rw[D + 1];
       }
-      dsmem_st2(dsmem_addr(recv_ml_s + (uint32_t)(rank * 8 + r) * 8u, owner), M, l);
+      __stcg(reinterpret_cast<float2 *>(part + r * PRS + D), make_float2(M, l));
     }
   }
-  cluster_sync_all();
-
-  // ---- reduce the slice this CTA owns, [rank * per, (rank + 1) * per), over the S partials and write it: one
-  // warp per query row of the slice; lane s holds the statistics of partial s; the lanes form 4 groups that each
-  // sum every fourth partial for 8 x 4 channels, and the groups are added with shuffles ----
-  const int lo = rank * per, hi = lo + per;
-  for (int r = lo / D + warp; r * D < hi; r += NCW + 1) {
-    const int e0 = max(lo, r * D), e1 = min(hi, (r + 1) * D);
-    const float ms = lane < S ? recv_ml[(lane * 8 + r) * 2] : -INFINITY;
-    const float ls = lane < S ? recv_ml[(lane * 8 + r) * 2 + 1] : 0.f;
-    float M = ms;
-#pragma unroll
-    for (int sh = 16; sh >= 1; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
-    const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
-    float L = f * ls;
-#pragma unroll
-    for (int sh = 16; sh >= 1; sh >>= 1) L += __shfl_xor_sync(0xffffffffu, L, sh);
-    const float inv = L > 0.f ? 1.f / L : 0.f;   // an empty sequence gives zeros
-    const int grp = lane >> 3, l8 = lane & 7;
-    for (int base = e0; base < e1; base += 32) {
-      const int e = base + l8 * 4;
-      const bool valid = e < e1;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int k = 0; k < kMaxSplits / 4; ++k) {
-        const int sp = grp + 4 * k;
-        const float fs = __shfl_sync(0xffffffffu, f, sp);
-        if (sp < S && valid) {
-          const float4 x = *reinterpret_cast<const float4 *>(recv_o + sp * per + (e - lo));
-          acc.x = fmaf(fs, x.x, acc.x); acc.y = fmaf(fs, x.y, acc.y);
-          acc.z = fmaf(fs, x.z, acc.z); acc.w = fmaf(fs, x.w, acc.w);
-        }
-      }
-#pragma unroll
-      for (int sh = 8; sh <= 16; sh <<= 1) {
-        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, sh); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, sh);
-        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, sh); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, sh);
-      }
-      if (grp == 0 && valid) {
-        const __nv_bfloat162 p0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-        const __nv_bfloat162 p1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-        uint2 pk;
-        pk.x = *reinterpret_cast<const uint32_t *>(&p0);
-        pk.y = *reinterpret_cast<const uint32_t *>(&p1);
-        *reinterpret_cast<uint2 *>(a.out + qrow0 * D + e) = pk;
-      }
-    }
-    if (rec && e0 == r * D && lane == 0) reinterpret_cast<float2 *>(c.hist_ml)[hrow + r] = make_float2(M, L);
+  // ---- the last CTA of the segment to get here merges the partials and writes the output ----
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int tk = atomicAdd(&c.att_tickets[seg], 1);
+    s_last = tk == S - 1;
+    if (tk == S - 1) c.att_tickets[seg] = 0;
+  }
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    const int nact = min(S, (npages + pps - 1) / pps);   // CTAs that had pages (the first nact)
+    float2 *hist = rec ? reinterpret_cast<float2 *>(c.hist_ml) + hrow : nullptr;
+    if (G <= 4)
+      merge_partials<D, NCW + 1, 4, 4>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist);
+    else
+      merge_partials<D, NCW + 1, 8, 1>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist);
   }
   if (rec && rank == 0)   // the queries themselves: G rows of D bf16
     for (int i = tid; i < G * D / 8; i += blockDim.x)

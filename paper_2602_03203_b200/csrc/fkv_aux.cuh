@@ -13,6 +13,7 @@ __global__ void k_reset(Ctx c) {
   for (int i = t0; i < c.num_pages; i += stride) c.free_stack[i] = c.num_pages - 1 - i;
   for (int i = t0; i < c.L * c.batch; i += stride) c.len[i] = 0;
   for (int i = t0; i < c.L * c.batch; i += stride) c.seq_tickets[i] = 0;
+  for (int i = t0; i < c.L * c.batch * c.Hkv; i += stride) c.att_tickets[i] = 0;
   if (c.hist_w)
     for (int i = t0; i < c.L * c.batch; i += stride) c.hist_cnt[i] = 0;
   if (t0 == 0) {

@@ -62,6 +62,10 @@ struct Ctx {
   int *tile1_start;  // prefix of score tiles over the work list
   int *planhdr;
   int *seq_tickets;  // [L][batch]
+  // Split-K attention: partial results [L*batch*Hkv][att_smax][G][D + 4] fp32 and one arrival counter per segment.
+  float *att_part;
+  int *att_tickets;
+  int att_smax;
   // Record of the decode queries of the current chunk (attention-feature maintenance; hist_w = 0: off).
   int hist_w;          // ring capacity W in queries
   uint8_t *hist_q;     // [L][batch][W][Hkv * G][D] bf16
