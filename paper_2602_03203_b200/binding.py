@@ -54,6 +54,13 @@ def lib():
         for name in EXPORTS:
             getattr(_lib, name).restype = ctypes.c_int
         _lib.fkv_last_cuda_error.restype = ctypes.c_char_p
+        vp, i32, u64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint64, ctypes.c_float
+        # Declared argument types for the per-token calls: plain ints and floats are converted by ctypes itself.
+        _lib.fkv_append.argtypes = [vp, i32, vp, vp, vp, u64, vp]
+        _lib.fkv_decode_attn.argtypes = [vp, i32, vp, vp, f32, vp]
+        _lib.fkv_append_decode_attn.argtypes = [vp, i32, vp, vp, vp, u64, vp, vp, f32, vp]
+        _lib.fkv_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, f32, vp]
+        _lib.fkv_evict.argtypes = [vp, i32, vp]
     return _lib
 
 
@@ -63,15 +70,24 @@ def _check(code: int, where: str):
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None, device_type="cuda"):
+    """Address of a contiguous tensor on the expected device (NULL for None)."""
     if t is None:
         return ctypes.c_void_p(0)
-    assert t.is_contiguous() and t.device.type == device_type, (t.device, t.is_contiguous())
-    if dtype is not None:
-        assert t.dtype == dtype, (t.dtype, dtype)
+    if not t.is_contiguous() or t.is_cuda != (device_type == "cuda") or (dtype is not None and t.dtype is not dtype):
+        raise ValueError(f"expected a contiguous {dtype} tensor on {device_type}, got {t.dtype} on {t.device}, "
+                         f"contiguous={t.is_contiguous()}")
     return ctypes.c_void_p(t.data_ptr())
 
 
+try:   # the raw handle of torch's current stream without building a Stream object (a hot-path saving)
+    _raw_stream = torch._C._cuda_getCurrentRawStream
+except AttributeError:   # pragma: no cover
+    _raw_stream = None
+
+
 def _stream():
+    if _raw_stream is not None:
+        return ctypes.c_void_p(_raw_stream(torch.cuda.current_device()))
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
@@ -139,7 +155,7 @@ class Cache:
     # -- the four calls of the path
     def append(self, layer, k, v, pos=None, seq_mask=0):
         _check(lib().fkv_append(self._h, layer, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
-                                _ptr(pos, torch.int32), ctypes.c_uint64(seq_mask), _stream()), "fkv_append")
+                                _ptr(pos, torch.int32), seq_mask, _stream()), "fkv_append")
 
     def evict(self, layer=ALL_LAYERS):
         _check(lib().fkv_evict(self._h, layer, _stream()), "fkv_evict")
@@ -156,8 +172,8 @@ class Cache:
     def decode_attn(self, layer, q, out=None, scale=0.0):
         if out is None:
             out = torch.empty_like(q)
-        _check(lib().fkv_decode_attn(self._h, layer, _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16),
-                                     ctypes.c_float(scale), _stream()), "fkv_decode_attn")
+        _check(lib().fkv_decode_attn(self._h, layer, _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16), scale,
+                                     _stream()), "fkv_decode_attn")
         return out
 
     def append_decode_attn(self, layer, k, v, q, out=None, pos=None, seq_mask=0, scale=0.0):
@@ -165,9 +181,8 @@ class Cache:
         if out is None:
             out = torch.empty_like(q)
         _check(lib().fkv_append_decode_attn(self._h, layer, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
-                                            _ptr(pos, torch.int32), ctypes.c_uint64(seq_mask), _ptr(q, torch.bfloat16),
-                                            _ptr(out, torch.bfloat16), ctypes.c_float(scale), _stream()),
-               "fkv_append_decode_attn")
+                                            _ptr(pos, torch.int32), seq_mask, _ptr(q, torch.bfloat16),
+                                            _ptr(out, torch.bfloat16), scale, _stream()), "fkv_append_decode_attn")
         return out
 
     def decode_step(self, k, v, q, out=None, pos=None, scale=0.0):
@@ -175,8 +190,8 @@ class Cache:
         if out is None:
             out = torch.empty_like(q)
         _check(lib().fkv_decode_step(self._h, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16), _ptr(pos, torch.int32),
-                                     _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16), ctypes.c_float(scale),
-                                     _stream()), "fkv_decode_step")
+                                     _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16), scale, _stream()),
+               "fkv_decode_step")
         return out
 
     # -- staged entry points
