@@ -39,7 +39,12 @@
 // programmatic-dependent-launch attribute: its CTAs start as soon as layer
 // l-1's CTAs are all running and stream their pages while those still
 // compute (three CTAs fit on an SM, so consecutive launches are co-resident).
-// Without the attribute the launch is ordered like any other.
+// Without the attribute the launch is ordered like any other.  Since such a
+// grid starts while the one before it is still running, everything an earlier
+// launch may have written (lengths, page tables, free stack, the caller's
+// q / k / v) is read with L2-only loads (ld.global.cg), so that no L1 line
+// filled earlier can be involved; pages come through the bulk-copy engine,
+// which reads L2 as well.
 #pragma once
 #include "fkv_dev.cuh"
 
@@ -72,6 +77,7 @@ struct AttendArgs {
 // The CTA-wide barrier, for the place where the producer warp and the consumer warps meet from different branches.
 __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 0;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 // The merge of a segment's split partials, run by the whole CTA that finished last.  part: [nact][G][D + 4] fp32
 // (O relative to the partial's own maximum, then m and l); out: G rows of D bf16; scratch: shared memory,
 // NW * 8 * D + 16 floats.  One round trip to L2 per pass: warp w asks for partials w, w + NW, ... (PASS of them
@@ -189,10 +195,10 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   int ptv = 0, ptn = 0;
   if (warp == NCW) {
     const int e = rank * a.pps + lane;
-    if (e < c.max_pages) ptv = ptrow[e];
-    if (e + 32 < c.max_pages) ptn = ptrow[e + 32];
+    if (e < c.max_pages) ptv = __ldcg(ptrow + e);
+    if (e + 32 < c.max_pages) ptn = __ldcg(ptrow + e + 32);
   }
-  const int n_old = c.len[a.layer * c.batch + seq];
+  const int n_old = __ldcg(c.len + a.layer * c.batch + seq);
   // The host refuses an append past the capacity; a replayed launch (CUDA graph) is checked here instead.
   const bool want = a.append && (!a.seq_mask || ((a.seq_mask >> seq) & 1ull));
   const bool app = want && n_old < c.cap;
@@ -209,13 +215,14 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   const size_t qrow0 = ((size_t)seq * c.Hkv + head) * G;  // first query head of the group
   // Query record for the attention features: ring slot of this token in the (layer, sequence) history.
   const bool rec = app && c.hist_w > 0;
-  const int hcnt = rec ? c.hist_cnt[a.layer * c.batch + seq] : 0;
+  const int hcnt = rec ? __ldcg(c.hist_cnt + a.layer * c.batch + seq) : 0;
   const size_t hrow = ((size_t)(a.layer * c.batch + seq) * (rec ? c.hist_w : 1) + (rec ? hcnt % c.hist_w : 0)) * (c.Hkv * G) +
                       (size_t)head * G;   // first query head of the group in the record
 
   const size_t ring_bytes = AttendSmem::ring(D, NCW, SLOTS);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + ring_bytes);                      // full[SLOTS], empty[SLOTS]
   const int gid = lane >> 2, tig = lane & 3;
+  const uint32_t rt_zero = gridDim.z - 1;   // 0 at run time (the grid is two-dimensional), unknown at compile time
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // queries 2 tig and 2 tig + 1
   float o[MT][4];
 #pragma unroll
@@ -246,8 +253,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
     __syncwarp();
     // ptv / ptn: page ids of the CTA's pages [0, 32) and [32, 64), one per lane.
     if (active && pps != a.pps) {   // the early read looked in the wrong place
-      ptv = lane < npg ? ptrow[pg0 + lane] : 0;
-      ptn = 32 + lane < npg ? ptrow[pg0 + 32 + lane] : 0;
+      ptv = lane < npg ? __ldcg(ptrow + pg0 + lane) : 0;
+      ptn = 32 + lane < npg ? __ldcg(ptrow + pg0 + 32 + lane) : 0;
     }
     if (lane < SLOTS && lane < npg) issue(lane, ptv);         // the ring is empty: no wait
     cta_sync();
@@ -267,19 +274,19 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
             atomicAdd(&c.ctrl[CTRL_FREE_TOP], 1);
             set_status(c, kDevPoolExhausted);
           } else {
-            npid = c.free_stack[old - 1];
+            npid = __ldcg(c.free_stack + old - 1);
             ptrow[npages - 1] = npid;
           }
         }
         npid = __shfl_sync(0xffffffffu, npid, 0);
       } else {
-        npid = ptrow[npages - 1];
+        npid = __ldcg(ptrow + npages - 1);
       }
       if (npid >= 0) {
         int32_t pdef = 0;
         if (!a.pos_new && n_old > 0) {
-          const uint8_t *prev = c.pool + (size_t)ptrow[(n_old - 1) / kPage] * c.page_bytes;
-          pdef = reinterpret_cast<const int32_t *>(meta_row(c, prev, (n_old - 1) % kPage))[c.F] + 1;
+          const uint8_t *prev = c.pool + (size_t)__ldcg(ptrow + (n_old - 1) / kPage) * c.page_bytes;
+          pdef = __ldcg(reinterpret_cast<const int32_t *>(meta_row(c, prev, (n_old - 1) % kPage)) + c.F) + 1;
         }
         const size_t row = (size_t)seq * c.Hkv + head;
         move_row<0>(c, c.pool + (size_t)npid * c.page_bytes, n_old % kPage, const_cast<uint8_t *>(a.k_new) + row * D * 2,
@@ -294,7 +301,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
     for (int i = SLOTS; i < npg; i += NCW) {
       if ((i & 31) == 0) {
         ptv = ptn;
-        ptn = i + 32 + lane < npg ? ptrow[pg0 + i + 32 + lane] : 0;
+        ptn = i + 32 + lane < npg ? __ldcg(ptrow + pg0 + i + 32 + lane) : 0;
       }
       const int pid = __shfl_sync(0xffffffffu, ptv, (i + lane) & 31);
       bool ok = true;
@@ -315,8 +322,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
       const uint32_t *qr = reinterpret_cast<const uint32_t *>(a.q + (qrow0 + gid) * D);
 #pragma unroll
       for (int ks = 0; ks < KSQ; ++ks) {
-        qb[ks][0] = gid < G ? qr[ks * 8 + tig] : 0u;
-        qb[ks][1] = gid < G ? qr[ks * 8 + 4 + tig] : 0u;
+        qb[ks][0] = gid < G ? __ldcg(qr + ks * 8 + tig) : 0u;
+        qb[ks][1] = gid < G ? __ldcg(qr + ks * 8 + 4 + tig) : 0u;
       }
     }
     // The new pair, one 16-byte chunk per lane (K chunks, then V chunks), for the warp that gets its page.
@@ -325,7 +332,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
     if (mine_new && lane < 2 * NCH) {
       const size_t row = (size_t)seq * c.Hkv + head;
       const uint8_t *src = (lane < NCH ? a.k_new : a.v_new) + row * D * 2 + (lane % NCH) * 16;
-      newrow = *reinterpret_cast<const uint4 *>(src);
+      newrow = __ldcg(reinterpret_cast<const uint4 *>(src));
     }
     // ldmatrix lane roles.  K (plain): matrix lane/8 -> keys ((lane/8)&1)*8.., channel chunk +lane/16.
     // V (transposed): matrix lane/8 -> keys (lane/16)*8.., channel chunk +(lane/8)&1.
@@ -383,8 +390,14 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
         o[mt][0] *= c0; o[mt][1] *= c1; o[mt][2] *= c0; o[mt][3] *= c1;
         mma_bf16(o[mt], x[0], x[1], x[2], x[3], pb0, pb1);
       }
+      // The slot may be refilled as soon as the arrival below is seen, so every read of the page has to be
+      // complete before it: the barrier's address is made to depend on the results of all the V mma's (whose
+      // operands are the last fragments read from the page) through a zero the compiler cannot see through.
+      uint32_t done = 0;
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) done |= __float_as_uint(o[mt][0]);
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars[SLOTS + slot_i]));
+      if (lane == 0) mbar_arrive(smem_u32(&bars[SLOTS + slot_i]) + (done & rt_zero));
     }
 #pragma unroll
     for (int sh = 4; sh < 32; sh <<= 1) {
@@ -467,7 +480,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   }
   if (rec && rank == 0)   // the queries themselves: G rows of D bf16
     for (int i = tid; i < G * D / 8; i += blockDim.x)
-      reinterpret_cast<uint4 *>(c.hist_q + hrow * D * 2)[i] = reinterpret_cast<const uint4 *>(a.q + qrow0 * D)[i];
+      reinterpret_cast<uint4 *>(c.hist_q + hrow * D * 2)[i] = __ldcg(reinterpret_cast<const uint4 *>(a.q + qrow0 * D) + i);
 
   // ---- the length grows once every CTA of the sequence (all heads, all splits) has read the old one ----
   if (app && tid == 0) {
@@ -483,6 +496,12 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
       }
     }
   }
+  // A launch with the programmatic attribute starts without waiting for the launch before it; it must not be
+  // COMPLETE before that one is, or whatever is ordered after this grid (the next decode step, an eviction, the end
+  // of a recorded graph) would not be ordered after the whole chain.  One thread of the grid waits for the
+  // launch before (all its own work is done by now; without the attribute this returns at once); every other CTA
+  // leaves and frees its SM.
+  if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) griddep_wait();
 }
 
 }  // namespace fkv

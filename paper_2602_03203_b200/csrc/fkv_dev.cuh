@@ -197,6 +197,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // ---------------------------------------------------------------- row movers
 // One warp moves one pair (K row, V row, feature row, position) between a
 // dense row and a slot of a page record.  DIR 0: dense -> page, 1: page -> dense.
+// The dense side is read through L2 (callers may run alongside the launch before them, see k_attend).
 template <int DIR>
 __device__ __forceinline__ void move_row(const Ctx &c, uint8_t *page, int r, uint8_t *k, uint8_t *v, float *feat,
                                          int32_t *pos, int lane, int32_t pos_default) {
@@ -206,19 +207,19 @@ __device__ __forceinline__ void move_row(const Ctx &c, uint8_t *page, int r, uin
     uint4 *pp = reinterpret_cast<uint4 *>(page + (isv ? c.off_v : 0) + kv_chunk_off(r, ch, c.D));
     uint8_t *dense = isv ? v : k;
     if (DIR == 0) {
-      *pp = dense ? *reinterpret_cast<const uint4 *>(dense + ch * 16) : make_uint4(0, 0, 0, 0);
+      *pp = dense ? __ldcg(reinterpret_cast<const uint4 *>(dense + ch * 16)) : make_uint4(0, 0, 0, 0);
     } else if (dense) {
       *reinterpret_cast<uint4 *>(dense + ch * 16) = *pp;
     }
   }
   float *pf = meta_row(c, page, r);
   for (int f = lane; f < c.F; f += 32) {
-    if (DIR == 0) pf[f] = feat ? feat[f] : 0.f;
+    if (DIR == 0) pf[f] = feat ? __ldcg(feat + f) : 0.f;
     else if (feat) feat[f] = pf[f];
   }
   if (lane == 0) {
     int32_t *pp = reinterpret_cast<int32_t *>(pf + c.F);
-    if (DIR == 0) *pp = pos ? *pos : pos_default;
+    if (DIR == 0) *pp = pos ? __ldcg(pos) : pos_default;
     else if (pos) *pos = *pp;
   }
 }

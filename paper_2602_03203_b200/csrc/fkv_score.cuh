@@ -219,8 +219,10 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) k_score(Ctx c, float *out, 
     const float mine = lane < 8 ? lo : hi;
     const int slot = tin * TILE + warp * kPage + lane;
     if (lane < kPage && slot < n) st_f32_hint(out + (size_t)(seg - seg_base) * c.cap + slot, mine + b2, keep);
+    // The slot may be refilled as soon as this arrival is seen: tie it to the score, which depends on every value
+    // read from the page, through a zero the compiler cannot see through (the grid is one-dimensional).
     __syncwarp();
-    if (lane == 0) mbar_arrive(smem_u32(&bars[nslots + slot_i]));
+    if (lane == 0) mbar_arrive(smem_u32(&bars[nslots + slot_i]) + (__float_as_uint(mine) & (gridDim.y - 1)));
     if (++ks == spw) { ks = 0; ph ^= 1; }
   }
 }

@@ -104,3 +104,55 @@ def test_replay_past_capacity_is_skipped_and_flagged():
             ref, ref64 = oracle.attend(qb[0, s, h * g:(h + 1) * g], k2, v2)
             err = np.abs(bits_to_f64(og[0, s, h * g:(h + 1) * g]) - bits_to_f64(ref))
             assert (err <= np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64))).all()
+
+
+def test_overlapped_decode_steps_are_reproducible_at_full_occupancy():
+    """The decode step of the Qwen3-4B-shaped configuration at B = 8192 puts three CTAs of consecutive layers'
+    launches on every SM, and an engine refills the SAME k / v / q buffers before every token.  Three repeats
+    of the same eight tokens must agree bit for bit (a page slot released before its last read, or an input
+    read at the wrong time, shows up as a run-to-run difference), and sampled heads must match the oracle."""
+    import dataclasses
+    w = wl.config(3, budget=8192)
+    w = dataclasses.replace(w, lens=tuple(min(n, b) for n, b in zip(w.lens, w.budgets)))
+    L, T = w.num_layers, 8
+    pages = binding.pages_for(w, L, 64)
+    need = binding.workspace_bytes_for(w, L, num_pages=pages, max_tokens=max(w.lens) + 64)
+    free, _ = torch.cuda.mem_get_info()
+    if need * 2.5 > free:   # workspace, its snapshot and generator scratch
+        pytest.skip(f"needs {need * 2.5 / 1e9:.1f} GB of device memory")
+    cache = binding.from_workload(w, L, num_pages=pages, max_tokens=max(w.lens) + 64)
+    for l in range(L):
+        K, V, A, pos = wl.layer_inputs(w, l, 0, "cuda")
+        cache.prefill(l, 0, K, V, A, pos)
+    snap = cache.snapshot()
+    gen = torch.Generator(device="cuda")
+    kd = torch.empty((L, 1, w.num_kv_heads, w.head_dim), device="cuda", dtype=torch.bfloat16)
+    vd = torch.empty_like(kd)
+    qd = torch.empty((L, 1, w.num_q_heads, w.head_dim), device="cuda", dtype=torch.bfloat16)
+
+    def run():
+        cache.restore(snap)
+        gen.manual_seed(7)
+        outs, qs = [], []
+        for _ in range(T):
+            for buf in (kd, vd, qd):
+                buf.copy_(torch.randn(buf.shape, device="cuda", generator=gen))
+            outs.append(cache.decode_step(kd, vd, qd))
+            qs.append(qd.clone())
+        torch.cuda.synchronize()
+        return torch.stack(outs), torch.stack(qs)
+
+    first, qs = run()
+    for _ in range(2):
+        again, _ = run()
+        assert torch.equal(first, again)
+    assert cache.device_status()[0] == 0
+    g, n0 = w.group_size, w.lens[0]
+    ob, qb = bits(first), bits(qs)
+    for l, h in [(0, 0), (5, 3), (18, 5), (35, 7)]:
+        k2, v2, _, _ = (bits(x) if x.dtype == torch.bfloat16 else x for x in cache.export_head(l, 0, h))
+        for t in (0, 3, T - 1):
+            n = n0 + t + 1
+            ref, ref64 = oracle.attend(qb[t, l, 0, h * g:(h + 1) * g], k2[:n], v2[:n])
+            err = np.abs(bits_to_f64(ob[t, l, 0, h * g:(h + 1) * g]) - bits_to_f64(ref))
+            assert (err <= np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64))).all(), (l, h, t, err.max())
