@@ -246,3 +246,46 @@ def test_select_long_segments_bit_exact(n, B, R):
         ref = oracle.select(sc[0, h, :n], B, R)
         assert cnt[0, h] == len(ref) and np.array_equal(idx[0, h, :len(ref)], ref)
     assert c.device_status()[0] == 0
+
+
+def test_chunk_then_eviction_is_reproducible():
+    """Config 2's protocol on 8 layers: 24 decode tokens (overlapped launches, maintained features), then the
+    eviction, three times from the same state.  Every segment must end up with the same bytes each time: no step
+    may depend on how the launches happened to interleave."""
+    w = wl.config(2)
+    L, T = 8, 24
+    pages = binding.pages_for(w, L, 64)
+    cache = binding.from_workload(w, L, num_pages=pages, max_tokens=max(w.lens) + 64, feature_window=32)
+    for l in range(L):
+        W1, b1, W2, b2 = wl.scorer_params(w, l, "cuda")
+        cache.load_scorers(l, W1, b1, W2, b2)
+        K, V, A, pos = wl.layer_inputs(w, l, 0, "cuda")
+        cache.prefill(l, 0, K, V, A, pos)
+    snap = cache.snapshot()
+    gen = torch.Generator(device="cuda")
+    kd = torch.empty((L, 1, w.num_kv_heads, w.head_dim), device="cuda", dtype=torch.bfloat16)
+    vd = torch.empty_like(kd)
+    qd = torch.empty((L, 1, w.num_q_heads, w.head_dim), device="cuda", dtype=torch.bfloat16)
+
+    def run():
+        cache.restore(snap)
+        gen.manual_seed(11)
+        outs = []
+        for _ in range(T):
+            for buf in (kd, vd, qd):
+                buf.copy_(torch.randn(buf.shape, device="cuda", generator=gen))
+            outs.append(cache.decode_step(kd, vd, qd))
+        cache.evict()
+        torch.cuda.synchronize()
+        state = [tuple(x.clone() for x in cache.export_head(l, 0, h)) for l in range(L) for h in range(w.num_kv_heads)]
+        return torch.stack(outs), state
+
+    out0, st0 = run()
+    assert all(k.shape[0] == w.budgets[0] for k, _, _, _ in st0)
+    for _ in range(2):
+        out, st = run()
+        assert torch.equal(out0, out)
+        for a, b in zip(st0, st):
+            for x, y in zip(a, b):
+                assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
+    assert cache.device_status()[0] == 0
