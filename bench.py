@@ -291,6 +291,25 @@ def run_ours(args):
         ev[0].record(); cache.evict_sampled(noise); ev[1].record(); torch.cuda.synchronize()
         sampled_ms.append(ev[0].elapsed_time(ev[1]))
     sampled_ms = ranks.max(min(sampled_ms[1:]))
+    # The same decode tokens with one ordinary launch per layer (fkv_append_decode_attn), i.e. without letting the
+    # layers of a token overlap: what a model sees whose projections sit between the layers.
+    serial_ms = 0.0
+    if T:
+        Ts = min(T, 4)
+        views = [[(kd[t][l], vd[t][l], qd[t][l], od[t][l]) for l in range(L)] for t in range(Ts)]
+        serial = []
+        for _ in range(3):
+            cache.restore(snap); torch.cuda.synchronize()
+            if not chunk_mode:
+                cache.evict(); torch.cuda.synchronize()
+            ev[0].record()
+            for t in range(Ts):
+                for l in range(L):
+                    k_, v_, q_, o_ = views[t][l]
+                    cache.append_decode_attn(l, k_, v_, q_, o_)
+            ev[1].record(); torch.cuda.synchronize()
+            serial.append(ev[0].elapsed_time(ev[1]) / (Ts * L))
+        serial_ms = ranks.max(min(serial[1:]))
     status, _ = cache.device_status()
     assert status == 0, f"device status {status}"
 
@@ -335,6 +354,8 @@ def run_ours(args):
         "decode_attn_gbs": N * dec_bytes / (decode_ms * 1e-3) / 1e9 if T else 0.0,
         "decode_attn_frac_of_measured_peak": dec_bytes / (decode_ms * 1e-3) / 1e9 / peak if T else 0.0,
         "decode_us_per_layer_launch": 1e3 * decode_ms / (T * L) if T else 0.0,
+        "decode_serialised_us_per_layer_launch": 1e3 * serial_ms,
+        "decode_serialised_tokens_per_s": N * w.batch / (serial_ms * L * 1e-3) if serial_ms else 0.0,
         "decode_note": "attention side only (append + GQA attention, one launch per layer, layers of a token "
                        "overlap); no projections, MLP or sampling",
         "roofline": {"bound": "hbm", "kernel": f"k_{dom}", "achieved": achieved, "peak": peak, "unit": "GB/s",
