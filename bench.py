@@ -310,6 +310,32 @@ def run_ours(args):
             ev[1].record(); torch.cuda.synchronize()
             serial.append(ev[0].elapsed_time(ev[1]) / (Ts * L))
         serial_ms = ranks.max(min(serial[1:]))
+    # The decode step recorded once into a CUDA graph and replayed per token (fixed k / v / q buffers): the host
+    # launches one graph instead of one kernel per layer, which matters where the step is launch-bound.
+    graph_ms = 0.0
+    if T:
+        gk, gv, gq, go = kd[0].clone(), vd[0].clone(), qd[0].clone(), od[0].clone()
+        cache.restore(snap)
+        if not chunk_mode:
+            cache.evict()
+        torch.cuda.synchronize()
+        before = cache.snapshot()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            cache.decode_step(gk, gv, gq, go)
+        torch.cuda.synchronize()
+        reps = []
+        for _ in range(3):
+            cache.restore(before); torch.cuda.synchronize()
+            ev[0].record()
+            for t in range(T):
+                graph.replay()
+            ev[1].record(); torch.cuda.synchronize()
+            reps.append(ev[0].elapsed_time(ev[1]) / (T * L))
+        cache.sync_lengths()
+        graph_ms = ranks.max(min(reps[1:]))
     status, _ = cache.device_status()
     assert status == 0, f"device status {status}"
 
@@ -354,6 +380,8 @@ def run_ours(args):
         "decode_attn_gbs": N * dec_bytes / (decode_ms * 1e-3) / 1e9 if T else 0.0,
         "decode_attn_frac_of_measured_peak": dec_bytes / (decode_ms * 1e-3) / 1e9 / peak if T else 0.0,
         "decode_us_per_layer_launch": 1e3 * decode_ms / (T * L) if T else 0.0,
+        "decode_graph_us_per_layer_launch": 1e3 * graph_ms,
+        "decode_graph_tokens_per_s": N * w.batch / (graph_ms * L * 1e-3) if graph_ms else 0.0,
         "decode_serialised_us_per_layer_launch": 1e3 * serial_ms,
         "decode_serialised_tokens_per_s": N * w.batch / (serial_ms * L * 1e-3) if serial_ms else 0.0,
         "decode_note": "attention side only (append + GQA attention, one launch per layer, layers of a token "
