@@ -268,6 +268,16 @@ def test_attention_parity_lengths(n, g, D):
     assert ld.cache.device_status()[0] == 0
 
 
+@pytest.mark.parametrize("n,g", [(20000, 4), (20000, 8), (2049, 4), (513, 7)])
+def test_attention_single_segment_many_splits(n, g):
+    # One KV head of one sequence: the launch uses the largest split count (32 for long segments), so the merge
+    # sees a partial in every lane, CTAs without pages, and more partials than one pass per warp takes.
+    w = wl.Workload("attn1", 1, 1, g, 128, (n,), (1 << 20,), 0, 22, "normal")
+    ld = Loaded(w)
+    assert _attn_check(ld, 0) <= ATTN_TOL
+    assert ld.cache.device_status()[0] == 0
+
+
 @pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
 def test_attention_after_evict(cfg):
     w = small(cfg)
