@@ -17,6 +17,10 @@
  *     as void*); calls return without synchronising unless they say "syncs".
  *     Calls on one cache must be issued on ONE stream, or be ordered by the
  *     caller; two calls on one cache that overlap on the GPU race.
+ *   - Host threads: a handle keeps a host-side mirror of the lengths and is not
+ *     thread-safe; use one host thread per handle at a time.  The first launch
+ *     of each kernel in a process sets its attributes without a lock, so make
+ *     the first calls on a device from one thread.
  *   - The library never allocates device memory for a cache.  The caller owns
  *     one device workspace (fkv_workspace_bytes) and keeps it alive until
  *     fkv_destroy; per-call tensors (k, v, q, out, ...) are borrowed until the
