@@ -743,13 +743,9 @@ int fkv_launch_count(const fkv_cache *c, uint64_t *launches) {
 }
 
 static int golden_select_launch(const float *alpha, int T, int B, int L, int M, int32_t *kept, cudaStream_t st) {
-  int P = 1;
-  while (P < B) P <<= 1;
-  const size_t smem = (size_t)P * 8 + (size_t)B * 8;
-  if (B > 8192 || smem > kMaxSmem - 1024) return FKV_ERR_CAPACITY;
-  static SmemOptIn opt_in;
-  FKV_CUDA(opt_in.ensure(k_golden_select, smem));
-  k_golden_select<<<1, 1024, smem, st>>>(alpha, T, B, L, M, P, kept);
+  if (B > 8192) return FKV_ERR_CAPACITY;   // eight cache entries per thread
+  const size_t smem = (size_t)B * 4;
+  k_golden_select<<<1, 1024, smem, st>>>(alpha, T, B, L, M, kept);
   FKV_CUDA(cudaGetLastError());
   return FKV_OK;
 }
