@@ -95,7 +95,8 @@ class Cache:
     """One budgeted KV cache on the current CUDA device (see include/fkv.h for the semantics)."""
 
     def __init__(self, num_layers, num_kv_heads, group_size, head_dim, max_batch, budget, max_tokens_per_head,
-                 recent_keep=0, activation=ACT_RELU, num_pages=0, page_size=16, scorer_hidden=16, feature_window=0):
+                 recent_keep=0, activation=ACT_RELU, num_pages=0, page_size=16, scorer_hidden=16, feature_window=0,
+                 workspace=None):
         if not torch.cuda.is_available():
             raise RuntimeError("fkv needs a CUDA device; there is no CPU path")
         self.cfg = FkvConfig(num_layers, num_kv_heads, group_size, head_dim, max_batch, page_size, scorer_hidden,
@@ -103,8 +104,17 @@ class Cache:
         nbytes = ctypes.c_size_t(0)
         _check(lib().fkv_workspace_bytes(ctypes.byref(self.cfg), ctypes.byref(nbytes)), "fkv_workspace_bytes")
         self.workspace_bytes = nbytes.value
-        self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device="cuda")
+        # The caller may bring the workspace (a CUDA uint8 tensor of at least workspace_bytes + 255 bytes); the
+        # library only ever touches [base, base + workspace_bytes) of it.
+        if workspace is None:
+            workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device="cuda")
+        if workspace.dtype != torch.uint8 or not workspace.is_cuda or not workspace.is_contiguous():
+            raise ValueError("workspace must be a contiguous CUDA uint8 tensor")
+        self.workspace = workspace
         base = (self.workspace.data_ptr() + 255) // 256 * 256
+        if base + nbytes.value > self.workspace.data_ptr() + self.workspace.numel():
+            raise ValueError(f"workspace too small: {self.workspace.numel()} bytes, need {nbytes.value} + alignment")
+        self.workspace_offset = base - self.workspace.data_ptr()
         self._h = ctypes.c_void_p(0)
         _check(lib().fkv_init_cache(ctypes.byref(self.cfg), ctypes.c_void_p(base), ctypes.c_size_t(nbytes.value),
                                     _stream(), ctypes.byref(self._h)), "fkv_init_cache")
@@ -334,12 +344,12 @@ def workspace_bytes_for(w, num_layers=None, num_pages=0, max_tokens=None) -> int
     return nbytes.value
 
 
-def from_workload(w, num_layers=None, num_pages=0, max_tokens=None, feature_window=0) -> Cache:
+def from_workload(w, num_layers=None, num_pages=0, max_tokens=None, feature_window=0, workspace=None) -> Cache:
     """A cache shaped for a ``workloads.Workload`` with per-sequence budgets set."""
     L = num_layers or w.num_layers
     c = Cache(L, w.num_kv_heads, w.group_size, w.head_dim, w.batch, max(w.budgets),
               max_tokens or (max(w.lens) + 256), recent_keep=w.recent_keep, activation=w.activation,
-              num_pages=num_pages, feature_window=feature_window)
+              num_pages=num_pages, feature_window=feature_window, workspace=workspace)
     for s, b in enumerate(w.budgets):
         if b != max(w.budgets):
             c.set_budget(s, b)

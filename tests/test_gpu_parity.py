@@ -526,3 +526,40 @@ def test_evict_sampled_zero_noise_equals_evict_and_short_noise_is_rejected():
     with pytest.raises(binding.FkvError) as e:
         c.cache.evict_sampled(torch.zeros((a.L, 1, w.num_kv_heads, 8), device="cuda"))
     assert e.value.code == -1
+
+
+# ------------------------------------------------------------------ the library stays inside its workspace
+def test_nothing_is_written_outside_the_workspace():
+    # A caller-owned buffer with guard zones before and after the workspace: a whole protocol run (prefill,
+    # decode steps with maintained features, deterministic and sampled evictions, staged calls, export) must
+    # leave every guard byte as it was.
+    w = small(2, num_layers=2, max_len=700)
+    guard = 1 << 20
+    cfg_probe = binding.from_workload(w, 2, max_tokens=max(w.lens) + 300, feature_window=32)
+    need = cfg_probe.workspace_bytes
+    cfg_probe.close()
+    buf = torch.full((guard + need + 512 + guard,), 0xA5, dtype=torch.uint8, device="cuda")
+    mid = buf[guard:guard + need + 512]
+    cache = binding.from_workload(w, 2, max_tokens=max(w.lens) + 300, feature_window=32, workspace=mid)
+    lo, hi = guard + cache.workspace_offset, guard + cache.workspace_offset + need
+    for l in range(2):
+        W1, b1, W2, b2 = wl.scorer_params(w, l)
+        cache.load_scorers(l, W1, b1, W2, b2)
+        K, V, A, pos = wl.layer_inputs(w, l, 0)
+        cache.prefill(l, 0, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
+    for step in range(40):
+        ks = torch.stack([wl.new_kv(w, l, step)[0] for l in range(2)]).cuda()
+        vs = torch.stack([wl.new_kv(w, l, step)[1] for l in range(2)]).cuda()
+        qs = torch.stack([wl.queries(w, l, step) for l in range(2)]).cuda()
+        cache.decode_step(ks, vs, qs)
+        if step == 19:
+            cache.evict()
+    n = cache.lengths(0)[0]
+    stride = 2 * max(1, n - w.budgets[0])
+    noise = torch.stack([wl.gumbel_noise(w, l, stride, device="cuda") for l in range(2)])
+    cache.evict_sampled(noise)
+    cache.score(0)
+    cache.export_head(1, 0, 0)
+    torch.cuda.synchronize()
+    assert cache.device_status()[0] == 0
+    assert bool((buf[:lo] == 0xA5).all()) and bool((buf[hi:] == 0xA5).all())
