@@ -421,62 +421,99 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   }
   __syncthreads();
 
-  // ---- this CTA's partial, relative to its own maximum, goes to global memory (it stays in L2): per query row
-  // D floats of O, then m and l ----
-  constexpr int PRS = D + 4;   // floats per row of a partial record
-  float *seg_part = c.att_part + (size_t)seg * c.att_smax * G * PRS;
-  if (active) {
-    float *part = seg_part + (size_t)rank * G * PRS;
+  if (S == 1) {
+    // ---- one CTA holds the whole segment (many segments per launch, or a short one): normalise and write the
+    // output straight from the warps' partials; nothing goes through global memory and no ticket is taken ----
     if (warp < NCW) {
       for (int e = tid * 4; e < G * D; e += NCW * 32 * 4) {
         const int r = e / D, ch = e - r * D;
-        float mw[NCW], M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < NCW; ++w) {
-          mw[w] = mg[((size_t)w * 8 + r) * MGS + D];
-          M = fmaxf(M, mw[w]);
-        }
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float M = -INFINITY, Lr = 0.f;
+        if (active) {
+          float mw[NCW];
 #pragma unroll
-        for (int w = 0; w < NCW; ++w) {
-          const float f = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);
-          const float4 x = *reinterpret_cast<const float4 *>(mg + ((size_t)w * 8 + r) * MGS + ch);
-          acc.x = fmaf(f, x.x, acc.x); acc.y = fmaf(f, x.y, acc.y);
-          acc.z = fmaf(f, x.z, acc.z); acc.w = fmaf(f, x.w, acc.w);
+          for (int w = 0; w < NCW; ++w) {
+            mw[w] = mg[((size_t)w * 8 + r) * MGS + D];
+            M = fmaxf(M, mw[w]);
+          }
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) {
+            const float f = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);
+            const float *rw = mg + ((size_t)w * 8 + r) * MGS;
+            const float4 x = *reinterpret_cast<const float4 *>(rw + ch);
+            acc.x = fmaf(f, x.x, acc.x); acc.y = fmaf(f, x.y, acc.y);
+            acc.z = fmaf(f, x.z, acc.z); acc.w = fmaf(f, x.w, acc.w);
+            Lr = fmaf(f, rw[D + 1], Lr);
+          }
         }
-        __stcg(reinterpret_cast<float4 *>(part + r * PRS + ch), acc);
+        const float inv = Lr > 0.f ? 1.f / Lr : 0.f;   // an empty sequence gives zeros
+        const __nv_bfloat162 p0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+        const __nv_bfloat162 p1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t *>(&p0);
+        pk.y = *reinterpret_cast<const uint32_t *>(&p1);
+        *reinterpret_cast<uint2 *>(a.out + (qrow0 + r) * D + ch) = pk;
+        if (rec && ch == 0) reinterpret_cast<float2 *>(c.hist_ml)[hrow + r] = make_float2(M, Lr);
       }
-    } else if (lane < G) {
-      const int r = lane;
-      float M = -INFINITY, l = 0.f;
-#pragma unroll
-      for (int w = 0; w < NCW; ++w) M = fmaxf(M, mg[((size_t)w * 8 + r) * MGS + D]);
-#pragma unroll
-      for (int w = 0; w < NCW; ++w) {
-        const float *rw = mg + ((size_t)w * 8 + r) * MGS;
-        l += (rw[D] == -INFINITY ? 0.f : exp2f(rw[D] - M)) * rw[D + 1];
-      }
-      __stcg(reinterpret_cast<float2 *>(part + r * PRS + D), make_float2(M, l));
     }
-  }
-  // ---- the last CTA of the segment to get here merges the partials and writes the output ----
-  __shared__ int s_last;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int tk = atomicAdd(&c.att_tickets[seg], 1);
-    s_last = tk == S - 1;
-    if (tk == S - 1) c.att_tickets[seg] = 0;
-  }
-  __syncthreads();
-  if (s_last) {
+  } else {
+    // ---- this CTA's partial, relative to its own maximum, goes to global memory (it stays in L2): per query row
+    // D floats of O, then m and l ----
+    constexpr int PRS = D + 4;   // floats per row of a partial record
+    float *seg_part = c.att_part + (size_t)seg * c.att_smax * G * PRS;
+    if (active) {
+      float *part = seg_part + (size_t)rank * G * PRS;
+      if (warp < NCW) {
+        for (int e = tid * 4; e < G * D; e += NCW * 32 * 4) {
+          const int r = e / D, ch = e - r * D;
+          float mw[NCW], M = -INFINITY;
+  #pragma unroll
+          for (int w = 0; w < NCW; ++w) {
+            mw[w] = mg[((size_t)w * 8 + r) * MGS + D];
+            M = fmaxf(M, mw[w]);
+          }
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  #pragma unroll
+          for (int w = 0; w < NCW; ++w) {
+            const float f = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);
+            const float4 x = *reinterpret_cast<const float4 *>(mg + ((size_t)w * 8 + r) * MGS + ch);
+            acc.x = fmaf(f, x.x, acc.x); acc.y = fmaf(f, x.y, acc.y);
+            acc.z = fmaf(f, x.z, acc.z); acc.w = fmaf(f, x.w, acc.w);
+          }
+          __stcg(reinterpret_cast<float4 *>(part + r * PRS + ch), acc);
+        }
+      } else if (lane < G) {
+        const int r = lane;
+        float M = -INFINITY, l = 0.f;
+  #pragma unroll
+        for (int w = 0; w < NCW; ++w) M = fmaxf(M, mg[((size_t)w * 8 + r) * MGS + D]);
+  #pragma unroll
+        for (int w = 0; w < NCW; ++w) {
+          const float *rw = mg + ((size_t)w * 8 + r) * MGS;
+          l += (rw[D] == -INFINITY ? 0.f : exp2f(rw[D] - M)) * rw[D + 1];
+        }
+        __stcg(reinterpret_cast<float2 *>(part + r * PRS + D), make_float2(M, l));
+      }
+    }
+    // ---- the last CTA of the segment to get here merges the partials and writes the output ----
+    __shared__ int s_last;
     __threadfence();
-    const int nact = min(S, (npages + pps - 1) / pps);   // CTAs that had pages (the first nact)
-    float2 *hist = rec ? reinterpret_cast<float2 *>(c.hist_ml) + hrow : nullptr;
-    if (G <= 4)
-      merge_partials<D, NCW + 1, 4, 4>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist);
-    else
-      merge_partials<D, NCW + 1, 8, 1>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist);
+    __syncthreads();
+    if (tid == 0) {
+      const int tk = atomicAdd(&c.att_tickets[seg], 1);
+      s_last = tk == S - 1;
+      if (tk == S - 1) c.att_tickets[seg] = 0;
+    }
+    __syncthreads();
+    if (s_last) {
+      __threadfence();
+      const int nact = min(S, (npages + pps - 1) / pps);   // CTAs that had pages (the first nact)
+      float2 *hist = rec ? reinterpret_cast<float2 *>(c.hist_ml) + hrow : nullptr;
+      if (G <= 4)
+        merge_partials<D, NCW + 1, 4, 4>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist);
+      else
+        merge_partials<D, NCW + 1, 8, 1>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist);
+    }
   }
   if (rec && rank == 0)   // the queries themselves: G rows of D bf16
     for (int i = tid; i < G * D / 8; i += blockDim.x)
