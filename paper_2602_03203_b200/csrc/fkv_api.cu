@@ -191,12 +191,14 @@ int launch_score_any(fkv_cache *c, float *out, int seg_base, int tiles_bound, cu
 void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float *scores, int32_t *idx,
                    int32_t *kept_count, int seg_base, int fill_pages, float *prio, const float *noise, int noise_stride,
                    int noise_base, cudaStream_t st) {
-  // Variant by the longest segment: registers hold a whole segment up to 8192 (small CTAs, two per SM) or
-  // 32768 keys; longer segments stream their rounds from L2.
+  // Variant by the longest segment: registers hold a whole segment up to 2048 (256-thread CTAs, many per SM), 8192
+  // (two CTAs per SM) or 32768 keys; longer segments stream their rounds from L2.
 #define FKV_SEL(S, M, T, P) \
   k_select<S, M, T, P><<<nblocks, T, 0, st>>>(c->ctx, scores, idx, kept_count, seg_base, fill_pages, prio, noise, \
                                              noise_stride, noise_base)
-  if (max_old <= kSelSmallThreads * kSelSmallPerThread) {
+  if (max_old <= kSelTinyThreads * kSelTinyPerThread) {
+    if (mode == 0) FKV_SEL(true, 0, kSelTinyThreads, kSelTinyPerThread); else FKV_SEL(true, 1, kSelTinyThreads, kSelTinyPerThread);
+  } else if (max_old <= kSelSmallThreads * kSelSmallPerThread) {
     if (mode == 0) FKV_SEL(true, 0, kSelSmallThreads, kSelSmallPerThread); else FKV_SEL(true, 1, kSelSmallThreads, kSelSmallPerThread);
   } else if (max_old <= kSelRound) {
     if (mode == 0) FKV_SEL(true, 0, kSelThreads, 32); else FKV_SEL(true, 1, kSelThreads, 32);

@@ -24,6 +24,7 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 
 constexpr int kSelThreads = 1024;   // the large variant: 1024 threads x 32 keys = one round of 32768
 constexpr int kSelSmallThreads = 512, kSelSmallPerThread = 16;   // segments of <= 8192 competing pairs: two CTAs per SM
+constexpr int kSelTinyThreads = 256, kSelTinyPerThread = 8;      // <= 2048 (budgets of 1K - 2K at large batch): many CTAs per SM
 
 // Fresh page ids of one compacted segment: copied from the batch the planner
 // reserved at the top of the free stack into the segment's row of pt_new.
