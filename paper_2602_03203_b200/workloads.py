@@ -85,7 +85,7 @@ def _config4_lens(seed: int) -> Tuple[int, ...]:
 
 
 def config(idx: int, budget: int | None = None) -> Workload:
-    """The five benchmark configurations (1-based, as listed in the benchmark spec)."""
+    """The five benchmark configurations (1-based): tiny, Qwen3-4B at 8K and 32K, 7B batched, 8B long-decode."""
     if idx == 1:
         return Workload("cfg1_tiny", 1, 2, 4, 64, (512,), (budget or 256,), 0, 0, "normal")
     if idx == 2:

@@ -1,6 +1,6 @@
 """Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element.
 
-Tolerances (stated by the benchmark spec):
+Tolerances:
   scores          max abs error <= 1e-3 (fp32 accumulation of bf16 inputs vs fp64)
   selection       bit-exact given identical scores
   compaction      bit-exact rows and positions
