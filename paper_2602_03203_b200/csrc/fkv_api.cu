@@ -52,7 +52,7 @@ struct SmemOptIn {
 };
 
 struct Layout {
-  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, att_part, att_tickets, hist_q, hist_ml, hist_n, hist_cnt, total;
+  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, att_part, att_tickets, hist_q, hist_mp, hist_n, hist_cnt, total;
   int cap, max_pages, num_pages, page_bytes, F, att_smax, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
 };
 
@@ -109,8 +109,9 @@ Layout make_layout(const fkv_config &c) {
   L.att_part = take(nseg * L.att_smax * c.group_size * (D + 4) * 4);
   L.att_tickets = take(nseg * 4);
   const size_t ls = (size_t)c.num_layers * c.max_batch, W = (size_t)c.feature_window, Hq = (size_t)c.num_kv_heads * c.group_size;
-  L.hist_q = take(ls * W * Hq * D * 2);
-  L.hist_ml = take(ls * W * Hq * 8);
+  const size_t Wp = (W + 15) & ~(size_t)15;   // rows of one query tile
+  L.hist_q = take(ls * Wp * Hq * D * 2);
+  L.hist_mp = take(ls * Wp * Hq * 4);
   L.hist_n = take(ls * W * 4);
   L.hist_cnt = take(W ? ls * 4 : 0);
   L.total = off;
@@ -208,15 +209,19 @@ void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float
 #undef FKV_SEL
 }
 
-// Attention features of the segments on the work list (after a k_plan): grid (groups of 8 pages, work items).
+// Attention features of the segments on the work list (after a k_plan): one persistent CTA per SM, each a
+// contiguous range of the plan's 128-pair tiles.
 template <int D>
 int launch_features_t(fkv_cache *c, int max_old, int nwork_bound, float scale_log2, cudaStream_t st) {
-  const size_t smem = FeatSmem::bytes(D, c->lay.F, c->cfg.feature_window);
+  static_assert(kFeatPages == kScorePPS, "the feature kernel walks the plan's score tiles");
+  int na = 0, nq = 0;
+  FeatSmem::rings(D, c->cfg.group_size, c->cfg.feature_window, na, nq);
+  if (na < 1) return FKV_ERR_INVALID_ARG;
+  const size_t smem = FeatSmem::bytes(D, c->cfg.group_size, c->cfg.feature_window, na, nq);
   static SmemOptIn opt_in;
   FKV_CUDA(opt_in.ensure(k_features<D>, smem));
-  dim3 grid(((max_old + kPage - 1) / kPage + kFeatPages - 1) / kFeatPages, nwork_bound);
-  if (grid.x == 0 || grid.y == 0) return FKV_OK;
-  k_features<D><<<grid, 256, smem, st>>>(c->ctx, scale_log2);
+  if (max_old <= 0 || nwork_bound <= 0) return FKV_OK;
+  k_features<D><<<c->sm_count, kFeatThreads, smem, st>>>(c->ctx, scale_log2, na, nq);
   FKV_LAUNCHED(c);
   return FKV_OK;
 }
@@ -327,7 +332,7 @@ int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, voi
   x.work = (int *)(ws + L.work); x.tile1_start = (int *)(ws + L.tile1);
   x.seq_tickets = (int *)(ws + L.seq_tickets);
   x.att_part = (float *)(ws + L.att_part); x.att_tickets = (int *)(ws + L.att_tickets); x.att_smax = L.att_smax;
-  x.hist_w = cfg->feature_window; x.hist_q = ws + L.hist_q; x.hist_ml = (float *)(ws + L.hist_ml);
+  x.hist_w = cfg->feature_window; x.hist_q = ws + L.hist_q; x.hist_mp = (float *)(ws + L.hist_mp); x.hist_wp = (cfg->feature_window + 15) & ~15;
   x.hist_n = (int *)(ws + L.hist_n); x.hist_cnt = (int *)(ws + L.hist_cnt);
   c->h_len.assign((size_t)cfg->num_layers * cfg->max_batch, 0);
   c->h_budget.assign(cfg->max_batch, cfg->budget);

@@ -85,7 +85,7 @@ __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wa
 // any of them.  R = query rows handled (>= G), a compile-time bound that sizes the register arrays.
 template <int D, int NW, int R, int PASS>
 __device__ __forceinline__ void merge_partials(const float *part, int nact, int G, float *scratch, __nv_bfloat16 *out,
-                                               float2 *hist_ml) {
+                                               float *hist_mp, int hist_stride) {
   constexpr int PRS = D + 4;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
   float *red = scratch;               // [NW][8][D]: one partial sum per warp
@@ -147,7 +147,7 @@ __device__ __forceinline__ void merge_partials(const float *part, int nact, int 
       for (int sh = 16; sh >= 1; sh >>= 1) L += __shfl_xor_sync(0xffffffffu, L, sh);
       if (lane == 0 && r < G) {
         tot[r] = L > 0.f ? 1.f / L : 0.f;   // an empty sequence gives zeros
-        if (hist_ml) hist_ml[r] = make_float2(M, L);
+        if (hist_mp) hist_mp[(size_t)r * hist_stride] = M + log2f(L);
       }
     }
   }
@@ -216,8 +216,9 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   // Query record for the attention features: ring slot of this token in the (layer, sequence) history.
   const bool rec = app && c.hist_w > 0;
   const int hcnt = rec ? __ldcg(c.hist_cnt + a.layer * c.batch + seq) : 0;
-  const size_t hrow = ((size_t)(a.layer * c.batch + seq) * (rec ? c.hist_w : 1) + (rec ? hcnt % c.hist_w : 0)) * (c.Hkv * G) +
-                      (size_t)head * G;   // first query head of the group in the record
+  const int hslot = rec ? hcnt % c.hist_w : 0;
+  const size_t hhead = (size_t)(a.layer * c.batch + seq) * (c.Hkv * G) + (size_t)head * G;   // first query head of the group in the record
+  float *hist_mp = rec ? c.hist_mp + hhead * c.hist_wp + hslot : nullptr;                    // its statistic of this token; next head: + hist_wp
 
   const size_t ring_bytes = AttendSmem::ring(D, NCW, SLOTS);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + ring_bytes);                      // full[SLOTS], empty[SLOTS]
@@ -453,7 +454,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
         pk.x = *reinterpret_cast<const uint32_t *>(&p0);
         pk.y = *reinterpret_cast<const uint32_t *>(&p1);
         *reinterpret_cast<uint2 *>(a.out + (qrow0 + r) * D + ch) = pk;
-        if (rec && ch == 0) reinterpret_cast<float2 *>(c.hist_ml)[hrow + r] = make_float2(M, Lr);
+        if (rec && ch == 0) hist_mp[(size_t)r * c.hist_wp] = M + log2f(Lr);
       }
     }
   } else {
@@ -508,16 +509,18 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
     if (s_last) {
       __threadfence();
       const int nact = min(S, (npages + pps - 1) / pps);   // CTAs that had pages (the first nact)
-      float2 *hist = rec ? reinterpret_cast<float2 *>(c.hist_ml) + hrow : nullptr;
       if (G <= 4)
-        merge_partials<D, NCW + 1, 4, 4>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist);
+        merge_partials<D, NCW + 1, 4, 4>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist_mp, c.hist_wp);
       else
-        merge_partials<D, NCW + 1, 8, 1>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist);
+        merge_partials<D, NCW + 1, 8, 1>(seg_part, nact, G, reinterpret_cast<float *>(smem), a.out + qrow0 * D, hist_mp, c.hist_wp);
     }
   }
-  if (rec && rank == 0)   // the queries themselves: G rows of D bf16
-    for (int i = tid; i < G * D / 8; i += blockDim.x)
-      reinterpret_cast<uint4 *>(c.hist_q + hrow * D * 2)[i] = __ldcg(reinterpret_cast<const uint4 *>(a.q + qrow0 * D) + i);
+  if (rec && rank == 0)   // the queries themselves: G rows of D bf16, laid out as the feature kernel's operand tile
+    for (int i = tid; i < G * D / 8; i += blockDim.x) {
+      const int r = i / (D / 8), ch = i % (D / 8);
+      *reinterpret_cast<uint4 *>(c.hist_q + hist_q_off(hhead + r, ch, hslot, c.hist_wp, D)) =
+          __ldcg(reinterpret_cast<const uint4 *>(a.q + qrow0 * D) + i);
+    }
 
   // ---- the length grows once every CTA of the sequence (all heads, all splits) has read the old one ----
   if (app && tid == 0) {

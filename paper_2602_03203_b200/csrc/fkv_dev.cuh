@@ -68,8 +68,10 @@ struct Ctx {
   int att_smax;
   // Record of the decode queries of the current chunk (attention-feature maintenance; hist_w = 0: off).
   int hist_w;          // ring capacity W in queries
-  uint8_t *hist_q;     // [L][batch][W][Hkv * G][D] bf16
-  float *hist_ml;      // [L][batch][W][Hkv * G][2]: softmax max and sum of that query (log2 domain)
+  int hist_wp;         // W rounded up to a multiple of 16: the row count of one operand tile
+  uint8_t *hist_q;     // [L][batch][Hkv * G][D / 64][hist_wp][64] bf16: per query head the K-major operand tile of
+                       // the feature kernel (row = ring slot, 128-byte rows, chunks XOR-swizzled by the row)
+  float *hist_mp;      // [L][batch][Hkv * G][hist_wp]: log2 of the softmax denominator of that query, max included
   int *hist_n;         // [L][batch][W]: pairs the query saw
   int *hist_cnt;       // [L][batch]: queries recorded since the last eviction
 };
@@ -82,6 +84,13 @@ __device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head
 // follows the K row (+ 2D bytes).  Chunks are XOR-swizzled by the row index inside each 128-byte span.
 __device__ __forceinline__ int kv_chunk_off(int r, int ch, int D) {
   return r * (4 * D) + ((ch >> 3) << 7) + (((ch & 7) ^ (r & 7)) << 4);
+}
+
+// Byte offset, inside the query record, of 16-byte chunk `ch` of the query that head `qhead` (index over layer,
+// sequence and query head) issued at ring slot `slot`: one tile of wp rows x 128 bytes per 64 channels, the
+// chunks of a row XOR-swizzled by the row index like the K rows of a page record.
+__device__ __forceinline__ size_t hist_q_off(size_t qhead, int ch, int slot, int wp, int D) {
+  return ((qhead * (D / 64) + (ch >> 3)) * wp + slot) * 128 + (size_t)(((ch & 7) ^ (slot & 7)) << 4);
 }
 
 // Meta row of pair r of a page record: F feature floats, then the position id.
