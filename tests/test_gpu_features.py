@@ -64,6 +64,55 @@ def test_update_features_matches_oracle(g, D, W, steps):
     assert c.device_status()[0] == 0
 
 
+@pytest.mark.parametrize("g,D,W,hkv,lens", [
+    # all four heads' records resident, four accumulators, four 32-query chunks per row, 4 tiles per CTA
+    (4, 128, 128, 4, (2700, 2300, 2500, 1900, 2900, 2100)),
+    # more than 128 queries: two accumulators shared by two warpgroups each, records streamed per tile
+    (4, 128, 256, 4, (1300, 1100, 1500, 900, 1250, 1400, 1000, 1350)),
+    # odd group (the last head of a tile is multiplied alone), narrow accumulators
+    (7, 128, 64, 2, (5100, 4700, 5300, 4900)),
+    # head_dim 64, three chunks per row
+    (4, 64, 96, 4, (2600, 2200, 3000, 2400, 2800)),
+])
+def test_update_features_many_tiles(g, D, W, hkv, lens):
+    # Enough tiles that every CTA of the feature kernel walks several of them, crosses segment and sequence
+    # boundaries and reuses its shared-memory stages and tensor-memory accumulators; W recorded queries (a whole
+    # number of 32-query chunks, ring not wrapped), so all tiles but the last of a segment take the unmasked path.
+    w = wl.Workload("featbig", 1, hkv, g, D, lens, (1 << 20,) * len(lens), 0, 54, "normal")
+    c = binding.from_workload(w, 1, feature_window=W, max_tokens=max(lens) + W + 16)
+    c.load_scorers(0, *wl.scorer_params(w, 0))
+    st = {}
+    for s in range(w.batch):
+        K, V, A, pos = wl.layer_inputs(w, 0, s)
+        c.prefill(0, s, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
+        for h in range(hkv):
+            n = lens[s]
+            Kf = np.zeros((n + W, D), np.uint16); Kf[:n] = bits(K)[h]
+            Af = np.zeros((n + W, 6 * g), np.float32); Af[:n] = npf(A)[h]
+            st[(s, h)] = dict(K=Kf, A=Af, q=np.zeros((W, g, D), np.uint16), n=n)
+    for step in range(W):
+        k, v = wl.new_kv(w, 0, step)
+        q = wl.queries(w, 0, step)
+        c.append_decode_attn(0, k.cuda(), v.cuda(), q.cuda())
+        kb, qb = bits(k), bits(q)
+        for (s, h), d in st.items():
+            d["K"][d["n"] + step] = kb[s, h]
+            d["q"][step] = qb[s, h * g:(h + 1) * g]
+    c.update_features(0)
+    assert c.device_status()[0] == 0
+    # a sample of segments: first, last, and those in between where CTA ranges change segment
+    keys = sorted(st.keys())
+    for (s, h) in keys[::max(1, len(keys) // 9)] + [keys[-1]]:
+        d = st[(s, h)]
+        nv = (d["n"] + 1 + np.arange(W)).astype(np.int32)
+        exp = oracle.features(d["K"], d["q"], nv, d["A"])
+        _, _, a2, _ = c.export_head(0, s, h)
+        got = npf(a2)
+        assert got.shape == exp.shape
+        bad = np.abs(got - exp) > FEAT_ATOL + FEAT_RTOL * np.abs(exp)
+        assert not bad.any(), (s, h, np.argwhere(bad)[:4], np.abs(got - exp).max())
+
+
 def test_no_recorded_query_leaves_features_alone():
     w = wl.Workload("feat0", 1, 2, 4, 128, (200,), (100,), 0, 52, "normal")
     c, st = _run_chunk(w, 32, 0)
