@@ -168,6 +168,7 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
 // The walk of one role over the CTA's tiles: which work item a tile is in and what that item's query record holds.
 struct FeatWalk {
   int wi, tbeg, tend, seg, n, ls, head, cnt, Lc, Lq, oldest_seen, newest;
+  bool ordered;   // ring not wrapped, whole 32-query chunks, and every query saw exactly one pair more than the one before
   float inv_Lc;
 };
 // A ring position and the phase bit of its barriers.  Kept by counting: the special-function pipe that an integer
@@ -178,7 +179,7 @@ struct FeatRing {
 };
 struct FeatTile {
   int pg0, np;
-  bool fast, first, last;
+  bool fast, masked, first, last;
 };
 // Tile t of the flat tile list; false if its segment has no query on record (its stored features stand).
 __device__ __forceinline__ bool feat_tile(const Ctx &c, int t, int t0, int t1, FeatWalk &w, FeatTile &x) {
@@ -194,6 +195,8 @@ __device__ __forceinline__ bool feat_tile(const Ctx &c, int t, int t0, int t1, F
     w.oldest_seen = w.Lc ? c.hist_n[(size_t)w.ls * c.hist_w + (w.cnt - w.Lc) % c.hist_w] : 0;
     w.newest = w.Lc ? (w.cnt - 1) % c.hist_w : 0;   // ring slot of the most recent query
     w.inv_Lc = w.Lc ? 1.f / (float)w.Lc : 0.f;
+    w.ordered = w.Lc > 0 && w.cnt <= c.hist_w && (w.Lc & 31) == 0 &&
+                c.hist_n[(size_t)w.ls * c.hist_w + w.newest] - w.oldest_seen == w.Lc - 1;
   }
   if (w.Lc == 0) return false;
   x.pg0 = (t - w.tbeg) * kFeatPages;
@@ -201,6 +204,9 @@ __device__ __forceinline__ bool feat_tile(const Ctx &c, int t, int t0, int t1, F
   // No masks needed: every recorded query saw the whole tile (the oldest one saw the fewest pairs), the ring has
   // not wrapped (slot order = time order) and the record is whole 32-column chunks.
   x.fast = x.pg0 * kPage + kFeatPages * kPage <= w.oldest_seen && w.cnt <= c.hist_w && (w.Lc & 31) == 0;
+  // Pairs appended during the chunk, but slot order = time order and query t saw the pairs below oldest_seen + t:
+  // a pair counts from one column on, a threshold per thread.
+  x.masked = !x.fast && w.ordered;
   x.first = t == w.tbeg || t == t0;         // first / last tile of its segment in this CTA's range
   x.last = t + 1 == w.tend || t + 1 == t1;
   return true;
@@ -215,6 +221,23 @@ __device__ __forceinline__ void feat_chunk(const uint32_t (&r)[32], const float 
     const float4 M4 = *reinterpret_cast<const float4 *>(mp + i);
     run += (ex2(fmaf(__uint_as_float(r[i + 3]), scale_log2, -M4.w)) + ex2(fmaf(__uint_as_float(r[i + 2]), scale_log2, -M4.z))) +
            (ex2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -M4.y)) + ex2(fmaf(__uint_as_float(r[i]), scale_log2, -M4.x)));
+    if (NEWEST && i == 24) w8 = run;
+    if (NEWEST && i == 16) w16 = run;
+  }
+}
+
+// The same for a pair that the queries before column `first` (relative to the chunk) did not see yet.
+template <bool NEWEST>
+__device__ __forceinline__ void feat_chunk_from(const uint32_t (&r)[32], const float *mp, float scale_log2, int first,
+                                                float &run, float &w8, float &w16) {
+#pragma unroll
+  for (int i = 28; i >= 0; i -= 4) {
+    const float4 M4 = *reinterpret_cast<const float4 *>(mp + i);
+    const float p3 = i + 3 >= first ? ex2(fmaf(__uint_as_float(r[i + 3]), scale_log2, -M4.w)) : 0.f;
+    const float p2 = i + 2 >= first ? ex2(fmaf(__uint_as_float(r[i + 2]), scale_log2, -M4.z)) : 0.f;
+    const float p1 = i + 1 >= first ? ex2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -M4.y)) : 0.f;
+    const float p0 = i >= first ? ex2(fmaf(__uint_as_float(r[i]), scale_log2, -M4.x)) : 0.f;
+    run += (p3 + p2) + (p1 + p0);
     if (NEWEST && i == 24) w8 = run;
     if (NEWEST && i == 16) w16 = run;
   }
@@ -403,7 +426,7 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
         frow = reinterpret_cast<float *>(c.pool + (size_t)c.pt[(size_t)w.seg * c.max_pages + x.pg0 + R / kPage] * c.page_bytes +
                                          c.off_f) + (R % kPage) * (c.F + 1);
       // 32-column chunks, counted from the newest: this warpgroup's are [k0, k1)
-      const int nch = (x.fast ? w.Lc : ((w.Lq + 31) & ~31)) >> 5, top = (nch - 1) << 5;
+      const int nch = ((w.Lq + 31) & ~31) >> 5, top = (nch - 1) << 5;   // (Lq = Lc on the two ordered paths)
       const int k0 = half == 0 ? 0 : (nch + 1) >> 1, k1 = (shared_acc && half == 0) ? (nch + 1) >> 1 : nch;
       for (int j = 0; j < G; ++j, ++u) {
         const int ss = resident ? sseg.i * G + j : sr.i, sp = resident ? sseg.ph : sr.ph;   // the head's statistics
@@ -432,6 +455,24 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
               w32 = run;
             } else {
               feat_chunk<false>(v, mp + a0, scale_log2, run, w8, w16);
+            }
+          }
+        } else if (x.masked) {
+          // Time order, but the pair is younger than some of the queries: it counts from column c0 on.  Chunks
+          // older than the warp's first pair's threshold (the smallest of the warp) hold nothing for any lane.
+          const int c0 = min(max(slot + 1 - w.oldest_seen, 0), w.Lc);
+          const int c0_warp = __shfl_sync(0xffffffffu, c0, 0);
+          for (int k = k0; k < k1; ++k) {
+            const int a0 = top - (k << 5);
+            if (a0 + 32 <= c0_warp) break;
+            uint32_t v[32];
+            tmem_ld32_issue(trow + (uint32_t)a0, v);
+            tmem_ld_wait(v);
+            if (k == 0) {
+              feat_chunk_from<true>(v, mp + a0, scale_log2, c0 - a0, run, w8, w16);
+              w32 = run;
+            } else {
+              feat_chunk_from<false>(v, mp + a0, scale_log2, c0 - a0, run, w8, w16);
             }
           }
         } else {
