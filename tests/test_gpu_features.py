@@ -64,22 +64,28 @@ def test_update_features_matches_oracle(g, D, W, steps):
     assert c.device_status()[0] == 0
 
 
-@pytest.mark.parametrize("g,D,W,hkv,lens", [
+@pytest.mark.parametrize("g,D,W,hkv,lens,steps", [
     # all four heads' records resident, four accumulators, four 32-query chunks per row, 4 tiles per CTA
-    (4, 128, 128, 4, (2700, 2300, 2500, 1900, 2900, 2100)),
+    (4, 128, 128, 4, (2700, 2300, 2500, 1900, 2900, 2100), 128),
     # more than 128 queries: two accumulators shared by two warpgroups each, records streamed per tile
-    (4, 128, 256, 4, (1300, 1100, 1500, 900, 1250, 1400, 1000, 1350)),
+    (4, 128, 256, 4, (1300, 1100, 1500, 900, 1250, 1400, 1000, 1350), 256),
     # odd group (the last head of a tile is multiplied alone), narrow accumulators
-    (7, 128, 64, 2, (5100, 4700, 5300, 4900)),
+    (7, 128, 64, 2, (5100, 4700, 5300, 4900), 64),
     # head_dim 64, three chunks per row
-    (4, 64, 96, 4, (2600, 2200, 3000, 2400, 2800)),
+    (4, 64, 96, 4, (2600, 2200, 3000, 2400, 2800), 96),
+    # one and two heads per group: a statistics slot is reused only after several segments
+    (1, 128, 64, 8, (1500, 700, 300, 1100, 200, 900), 64),
+    (2, 64, 32, 8, (1300, 500, 800, 1700, 150, 1000), 32),
+    # more tokens than the ring holds (slot order is not time order) and a partial last chunk: the general path
+    (4, 128, 64, 4, (2100, 1700, 2500, 1300), 90),
+    (4, 128, 128, 4, (2100, 1700, 2500, 1300), 50),
 ])
-def test_update_features_many_tiles(g, D, W, hkv, lens):
+def test_update_features_many_tiles(g, D, W, hkv, lens, steps):
     # Enough tiles that every CTA of the feature kernel walks several of them, crosses segment and sequence
-    # boundaries and reuses its shared-memory stages and tensor-memory accumulators; W recorded queries (a whole
-    # number of 32-query chunks, ring not wrapped), so all tiles but the last of a segment take the unmasked path.
+    # boundaries and reuses its shared-memory stages and tensor-memory accumulators.  With steps = W (a whole number
+    # of 32-query chunks, ring not wrapped) all tiles but the last of a segment take the unmasked path.
     w = wl.Workload("featbig", 1, hkv, g, D, lens, (1 << 20,) * len(lens), 0, 54, "normal")
-    c = binding.from_workload(w, 1, feature_window=W, max_tokens=max(lens) + W + 16)
+    c = binding.from_workload(w, 1, feature_window=W, max_tokens=max(lens) + steps + 16)
     c.load_scorers(0, *wl.scorer_params(w, 0))
     st = {}
     for s in range(w.batch):
@@ -87,10 +93,10 @@ def test_update_features_many_tiles(g, D, W, hkv, lens):
         c.prefill(0, s, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
         for h in range(hkv):
             n = lens[s]
-            Kf = np.zeros((n + W, D), np.uint16); Kf[:n] = bits(K)[h]
-            Af = np.zeros((n + W, 6 * g), np.float32); Af[:n] = npf(A)[h]
-            st[(s, h)] = dict(K=Kf, A=Af, q=np.zeros((W, g, D), np.uint16), n=n)
-    for step in range(W):
+            Kf = np.zeros((n + steps, D), np.uint16); Kf[:n] = bits(K)[h]
+            Af = np.zeros((n + steps, 6 * g), np.float32); Af[:n] = npf(A)[h]
+            st[(s, h)] = dict(K=Kf, A=Af, q=np.zeros((steps, g, D), np.uint16), n=n)
+    for step in range(steps):
         k, v = wl.new_kv(w, 0, step)
         q = wl.queries(w, 0, step)
         c.append_decode_attn(0, k.cuda(), v.cuda(), q.cuda())
@@ -104,8 +110,8 @@ def test_update_features_many_tiles(g, D, W, hkv, lens):
     keys = sorted(st.keys())
     for (s, h) in keys[::max(1, len(keys) // 9)] + [keys[-1]]:
         d = st[(s, h)]
-        nv = (d["n"] + 1 + np.arange(W)).astype(np.int32)
-        exp = oracle.features(d["K"], d["q"], nv, d["A"])
+        nv = (d["n"] + 1 + np.arange(steps)).astype(np.int32)
+        exp = oracle.features(d["K"], d["q"][-W:], nv[-W:], d["A"])     # the ring keeps the last W queries
         _, _, a2, _ = c.export_head(0, s, h)
         got = npf(a2)
         assert got.shape == exp.shape
