@@ -361,7 +361,8 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
       if (!mbar_spin(smem_u32(&a_full[sa]), pa)) { set_status(c, kDevWaitTimeout); break; }
       if (x.first) ++segs;
       const uint32_t idesc = umma_idesc_bf16(ROWS, w.Lq);
-      const uint32_t a0 = smem_u32(At + (size_t)sa * abytes);
+      const uint64_t ad0 = umma_desc_sw128(smem_u32(At + (size_t)sa * abytes));
+      const uint32_t qhalf16 = (uint32_t)(Lw * 128) >> 4;   // a 64-channel half of a record's tile, in 16-byte units
       // Two heads at a time when two accumulators are to be had: their k-steps alternate, so that an mma never has
       // to wait for the one before it on the same accumulator.
       for (int j = 0; j < G && ok; j += 2) {
@@ -379,17 +380,20 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
         if (!ok) break;
         tc_fence_after();
         {
+          // This thread's instruction count is on the critical path (it shares its scheduler with four reducing
+          // warps): descriptors are built once and advanced by adding to their address field (16-byte units).
+          const uint64_t bd0 = umma_desc_sw128(smem_u32(Qt + (size_t)sq[0] * qbytes));
+          const uint64_t bd1 = umma_desc_sw128(smem_u32(Qt + (size_t)sq[1] * qbytes));
+          const uint32_t d0 = tmem_base + (uint32_t)bb[0] * ncols, d1 = tmem_base + (uint32_t)bb[1] * ncols;
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {        // K = 16 channels per instruction: 32 bytes inside the swizzled row
-            const uint64_t ad = umma_desc_sw128(a0 + (ks >> 2) * ROWS * 128 + (ks & 3) * 32);
-            const uint32_t koff = (uint32_t)((ks >> 2) * Lw * 128 + (ks & 3) * 32);
-            const uint64_t bd0 = umma_desc_sw128(smem_u32(Qt + (size_t)sq[0] * qbytes) + koff);
+            const uint64_t ad = ad0 + (uint64_t)(((ks >> 2) * ROWS * 128 + (ks & 3) * 32) >> 4);
+            const uint64_t kb = (uint64_t)((ks >> 2) * qhalf16 + (ks & 3) * 2);
             if (nh == 2) {
-              const uint64_t bd1 = umma_desc_sw128(smem_u32(Qt + (size_t)sq[1] * qbytes) + koff);
-              umma_bf16_keep_a<true>(tmem_base + (uint32_t)bb[0] * ncols, ad, bd0, idesc, ks > 0);
-              umma_bf16_keep_a<false>(tmem_base + (uint32_t)bb[1] * ncols, ad, bd1, idesc, ks > 0);
+              umma_bf16_keep_a<true>(d0, ad, bd0 + kb, idesc, ks > 0);
+              umma_bf16_keep_a<false>(d1, ad, bd1 + kb, idesc, ks > 0);
             } else {
-              umma_bf16(tmem_base + (uint32_t)bb[0] * ncols, ad, bd0, idesc, ks > 0);
+              umma_bf16(d0, ad, bd0 + kb, idesc, ks > 0);
             }
           }
           for (int h = 0; h < nh; ++h) {
