@@ -425,10 +425,8 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
       if (x.first) sseg.next(SD);
       const int slot = x.pg0 * kPage + R;
       const bool live = half == 0 && slot < w.n;
-      float *frow = nullptr;
-      if (live)
-        frow = reinterpret_cast<float *>(c.pool + (size_t)c.pt[(size_t)w.seg * c.max_pages + x.pg0 + R / kPage] * c.page_bytes +
-                                         c.off_f) + (R % kPage) * (c.F + 1);
+      // The pair's page: asked for now, first used after the waits below (a use here would stall the warp at every tile).
+      const int pid = live ? c.pt[(size_t)w.seg * c.max_pages + x.pg0 + R / kPage] : 0;
       // 32-column chunks, counted from the newest: this warpgroup's are [k0, k1)
       const int nch = ((w.Lq + 31) & ~31) >> 5, top = (nch - 1) << 5;   // (Lq = Lc on the two ordered paths)
       const int k0 = half == 0 ? 0 : (nch + 1) >> 1, k1 = (shared_acc && half == 0) ? (nch + 1) >> 1 : nch;
@@ -437,14 +435,16 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
         if (!resident) sr.next(NS);
         const int b = u & (NB - 1);
         if (b != e) continue;
-        float old_sum = 0.f, old_dec = 0.f;
-        if (live) { old_sum = __ldcg(frow + j * 6 + 4); old_dec = __ldcg(frow + j * 6 + 5); }
         const float *mp = St + (size_t)ss * Lw;
         const uint32_t ph = (uint32_t)(u >> lgNB) & 1;
         if (!mbar_wait_warp(smem_u32(&s_full[ss]), sp) || !mbar_wait_warp(smem_u32(&acc_full[b]), ph)) {
           set_status(c, kDevWaitTimeout); ok = false; break;
         }
         tc_fence_after();
+        // The cumulative features to update: asked for here, used after the walk.
+        float *frow = reinterpret_cast<float *>(c.pool + (size_t)pid * c.page_bytes + c.off_f) + (R % kPage) * (c.F + 1);
+        float old_sum = 0.f, old_dec = 0.f;
+        if (live) { old_sum = __ldcg(frow + j * 6 + 4); old_dec = __ldcg(frow + j * 6 + 5); }
         const uint32_t trow = trow0 + (uint32_t)b * ncols;
         float run = 0.f, w8 = 0.f, w16 = 0.f, w32 = 0.f;
         if (x.fast) {
