@@ -49,7 +49,7 @@ def _expected(d, W):
 
 
 @pytest.mark.parametrize("g,D,W,steps", [(4, 128, 64, 40), (4, 128, 32, 45), (7, 128, 40, 40), (4, 64, 64, 33),
-                                         (1, 128, 16, 7), (8, 64, 24, 50)])
+                                         (1, 128, 16, 7), (8, 64, 24, 50), (2, 64, 8, 13), (4, 128, 8, 5)])
 def test_update_features_matches_oracle(g, D, W, steps):
     w = wl.Workload("feat", 2, 2, g, D, (100, 37), (1 << 20,) * 2, 0, 51, "normal")
     c, st = _run_chunk(w, W, steps)
