@@ -218,10 +218,16 @@ int launch_features_t(fkv_cache *c, int max_old, int nwork_bound, float scale_lo
   FeatSmem::rings(D, c->cfg.group_size, c->cfg.feature_window, na, nq);
   if (na < 1) return FKV_ERR_INVALID_ARG;
   const size_t smem = FeatSmem::bytes(D, c->cfg.group_size, c->cfg.feature_window, na, nq);
-  static SmemOptIn opt_in;
-  FKV_CUDA(opt_in.ensure(k_features<D>, smem));
   if (max_old <= 0 || nwork_bound <= 0) return FKV_OK;
-  k_features<D><<<c->sm_count, kFeatThreads, smem, st>>>(c->ctx, scale_log2, na, nq);
+  if (FeatSmem::lq(c->cfg.feature_window) <= 128) {   // four accumulators: three reducing warpgroups
+    static SmemOptIn opt_in;
+    FKV_CUDA(opt_in.ensure(k_features<D, 3>, smem));
+    k_features<D, 3><<<c->sm_count, feat_threads(3), smem, st>>>(c->ctx, scale_log2, na, nq);
+  } else {                                            // two accumulators, two warpgroups on each
+    static SmemOptIn opt_in;
+    FKV_CUDA(opt_in.ensure(k_features<D, 4>, smem));
+    k_features<D, 4><<<c->sm_count, feat_threads(4), smem, st>>>(c->ctx, scale_log2, na, nq);
+  }
   FKV_LAUNCHED(c);
   return FKV_OK;
 }

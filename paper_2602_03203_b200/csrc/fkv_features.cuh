@@ -23,8 +23,9 @@
 //     N = the padded query count, K = 16 per instruction) into one of four (two for more than 128
 //     queries) accumulators in tensor memory; tcgen05.commit hands the accumulator to a reducing warpgroup and the stages back to
 //     warp 0;
-//   - four warpgroups (warps 4-19) reduce, one accumulator each (with two accumulators, two
-//     warpgroups share one and split the query axis): a thread owns ONE pair (its tensor-memory
+//   - three warpgroups (warps 4-15) reduce, taking the units of the four accumulators in turn (with
+//     two accumulators there are four warpgroups, two share an accumulator and split the query
+//     axis): a thread owns ONE pair (its tensor-memory
 //     lane) and walks the query axis from the newest query back, 32 columns per tcgen05.ld: exp2,
 //     add; the windows 8 / 16 / 32 are prefixes of that walk.  The six features of the head go
 //     straight to the pair's meta row.
@@ -42,7 +43,10 @@ namespace fkv {
 constexpr float kFeatDecay = 0.9f;   // Appendix B.1: per-chunk decay of the decayed sum
 constexpr int kFeatPages = 8;        // pages (of 16 pairs) per tile: the M = 128 rows of the mma
 constexpr int kFeatMaxQueries = 256; // N of one mma; two accumulators of that width fill tensor memory
-constexpr int kFeatThreads = 640;    // warp 0: records, warp 1: mma, warps 2-3: K rows (warp 2 owns tensor memory), warps 4-19 reduce
+// warp 0: records, warp 1: mma, warps 2-3: K rows (warp 2 owns tensor memory), then WGS reducing warpgroups: four when
+// two of them share each of two accumulators (more than 128 queries), else three, which take the units of the four
+// accumulators in turn - 512 threads leave each 128 registers, and the reductions then need no spills.
+__host__ __device__ constexpr int feat_threads(int wgs) { return (4 + 4 * wgs) * 32; }
 constexpr int kFeatMaxA = 4, kFeatMaxQ = 8, kFeatMaxS = 24;   // ring depths the barrier block has room for
 
 struct FeatSmem {
@@ -243,8 +247,8 @@ __device__ __forceinline__ void feat_chunk_from(const uint32_t (&r)[32], const f
   }
 }
 
-template <int D>
-__global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale_log2, int NA, int NQ) {
+template <int D, int WGS>
+__global__ void __launch_bounds__(feat_threads(WGS), 1) k_features(Ctx c, float scale_log2, int NA, int NQ) {
   constexpr int HALVES = D / 64, ROWS = kFeatPages * kPage;   // 128 pairs
   extern __shared__ uint8_t smem_raw[];
   const int total = c.planhdr[PH_TILES1], nwork = c.planhdr[PH_NWORK];
@@ -417,7 +421,7 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
     const bool shared_acc = NB == 2;
     const int R = quarter * 32 + lane;
     const uint32_t trow0 = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    int u = 0;
+    int u = 0, u3 = 0;
     FeatRing sseg{SD - 1, 1}, sr{0, 0};
     bool ok = true;
     for (int t = t0; t < t1 && ok; ++t) {
@@ -425,8 +429,10 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
       if (x.first) sseg.next(SD);
       const int slot = x.pg0 * kPage + R;
       const bool live = half == 0 && slot < w.n;
-      // The pair's page: asked for now, first used after the waits below (a use here would stall the warp at every tile).
-      const int pid = live ? c.pt[(size_t)w.seg * c.max_pages + x.pg0 + R / kPage] : 0;
+      float *frow = nullptr;
+      if (live)
+        frow = reinterpret_cast<float *>(c.pool + (size_t)c.pt[(size_t)w.seg * c.max_pages + x.pg0 + R / kPage] * c.page_bytes +
+                                         c.off_f) + (R % kPage) * (c.F + 1);
       // 32-column chunks, counted from the newest: this warpgroup's are [k0, k1)
       const int nch = ((w.Lq + 31) & ~31) >> 5, top = (nch - 1) << 5;   // (Lq = Lc on the two ordered paths)
       const int k0 = half == 0 ? 0 : (nch + 1) >> 1, k1 = (shared_acc && half == 0) ? (nch + 1) >> 1 : nch;
@@ -434,17 +440,22 @@ __global__ void __launch_bounds__(kFeatThreads, 1) k_features(Ctx c, float scale
         const int ss = resident ? sseg.i * G + j : sr.i, sp = resident ? sseg.ph : sr.ph;   // the head's statistics
         if (!resident) sr.next(NS);
         const int b = u & (NB - 1);
-        if (b != e) continue;
+        if (WGS == 3) {   // three warpgroups: every third unit, whatever its accumulator
+          const bool mine = u3 == wg;
+          if (++u3 == 3) u3 = 0;
+          if (!mine) continue;
+        } else if (b != e) {
+          continue;
+        }
+        // The cumulative features to update: asked for here, used after the walk.
+        float old_sum = 0.f, old_dec = 0.f;
+        if (live) { old_sum = __ldcg(frow + j * 6 + 4); old_dec = __ldcg(frow + j * 6 + 5); }
         const float *mp = St + (size_t)ss * Lw;
         const uint32_t ph = (uint32_t)(u >> lgNB) & 1;
         if (!mbar_wait_warp(smem_u32(&s_full[ss]), sp) || !mbar_wait_warp(smem_u32(&acc_full[b]), ph)) {
           set_status(c, kDevWaitTimeout); ok = false; break;
         }
         tc_fence_after();
-        // The cumulative features to update: asked for here, used after the walk.
-        float *frow = reinterpret_cast<float *>(c.pool + (size_t)pid * c.page_bytes + c.off_f) + (R % kPage) * (c.F + 1);
-        float old_sum = 0.f, old_dec = 0.f;
-        if (live) { old_sum = __ldcg(frow + j * 6 + 4); old_dec = __ldcg(frow + j * 6 + 5); }
         const uint32_t trow = trow0 + (uint32_t)b * ncols;
         float run = 0.f, w8 = 0.f, w16 = 0.f, w32 = 0.f;
         if (x.fast) {
