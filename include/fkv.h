@@ -107,9 +107,14 @@ int fkv_reset(fkv_cache *c, void *stream);
  * Scorer of one (layer, KV head) - Appendix B.1:
  *   phi = sigma(x W1 + b1) W2 + b2,  x = Concat(k, v, a).
  * W1: host, [(2D+F)][H] row-major fp32, rows ordered k | v | a; b1, W2: host
- * [H].  The 2D rows of W1 that multiply k and v are stored as bf16 (round to
- * nearest even); the F feature rows, b1, W2, b2 stay fp32.  Copies to the
- * device on `stream` from a staging buffer the handle owns (syncs).
+ * [H].  The paper states no precision for the weights; they are taken as
+ * fp32.  The 2D rows of W1 that multiply k and v are stored as TWO bf16 values
+ * per weight, the rounding (to nearest even) of the weight and the rounding of
+ * the remainder, and both are multiplied with the bf16 channels on the tensor
+ * cores with fp32 accumulation: a weight enters with about 2^-17 relative
+ * error instead of bf16's 2^-9.  The F feature rows, b1, W2, b2 stay fp32.
+ * Copies to the device on `stream` from a staging buffer the handle owns
+ * (syncs).
  */
 int fkv_load_scorer(fkv_cache *c, int layer, int kv_head, const float *W1, const float *b1, const float *W2, float b2,
                     void *stream);

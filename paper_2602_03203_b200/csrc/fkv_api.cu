@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <cmath>
 #include <new>
 #include <string>
 #include <vector>
@@ -82,8 +83,8 @@ Layout make_layout(const fkv_config &c) {
   const int bpages = (std::min(c.budget, L.cap) + kPage - 1) / kPage;
   L.num_pages = c.num_pages ? c.num_pages : (int)std::min<size_t>(nseg * ((size_t)L.max_pages + bpages + 1), 0x7fffffff);
   const int KS = 2 * D / 16;
-  L.sp_off_wf = KS * 512;
-  L.sp_off_b1 = L.sp_off_wf + L.F * 64;
+  L.sp_off_wf = 2 * KS * 512;   // fragments of the roundings, then of the remainders
+  L.sp_off_b1 = L.sp_off_wf + ScoreSmem::fk(L.F) * 1024;   // feature rows: tf32 fragments, truncations and remainders
   L.sp_off_w2 = L.sp_off_b1 + 64;
   L.sp_off_b2 = L.sp_off_w2 + 64;
   L.sp_stride = (int)align_up((size_t)L.sp_off_b2 + 16, 256);
@@ -126,6 +127,13 @@ uint16_t f32_to_bf16_rne(float f) {
   return (uint16_t)(u >> 16);
 }
 
+float bf16_to_f32(uint16_t b) {
+  const uint32_t u = (uint32_t)b << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return f;
+}
+
 }  // namespace
 
 struct fkv_cache {
@@ -163,22 +171,24 @@ int cuda_fail(cudaError_t e) {
 
 bool layer_ok(const fkv_cache *c, int layer) { return layer >= 0 && layer < c->cfg.num_layers; }
 
-// Page slots per consumer warp of the scorer: as many as fit the shared memory, at most 4.
-int score_slots_per_warp(const fkv_cache *c) {
-  for (int spw = 4; spw >= 1; --spw)
-    if (ScoreSmem::bytes(c->lay.page_bytes, c->lay.F, kScorePPS, spw) <= kMaxSmem) return spw;
+// Page slots of the scorer's ring: as many as fit the shared memory, a multiple of the number of warps (a slot
+// must always come back to the warp that refilled it: its barrier carries one phase bit, and only the warp that
+// waited for the slot's previous page knows that phase is over), at most four per warp.
+int score_ring_slots(const fkv_cache *c) {
+  for (int n = 4 * kScorePPS; n >= kScorePPS; n -= kScorePPS)
+    if (ScoreSmem::bytes(c->lay.page_bytes, c->lay.F, kScorePPS, n) <= kMaxSmem) return n;
   return 0;
 }
 
 template <int D>
 int launch_score(fkv_cache *c, float *out, int seg_base, int tiles_bound, cudaStream_t st) {
-  const int spw = score_slots_per_warp(c);
-  if (spw == 0) return FKV_ERR_INVALID_ARG;
-  const size_t smem = ScoreSmem::bytes(c->lay.page_bytes, c->lay.F, kScorePPS, spw);
+  const int nslots = score_ring_slots(c);
+  if (nslots == 0) return FKV_ERR_INVALID_ARG;
+  const size_t smem = ScoreSmem::bytes(c->lay.page_bytes, c->lay.F, kScorePPS, nslots);
   static SmemOptIn opt_in;
   FKV_CUDA(opt_in.ensure(k_score<D, kScorePPS>, kMaxSmem));
   const int grid = std::max(1, std::min(c->sm_count, tiles_bound));
-  k_score<D, kScorePPS><<<grid, (kScorePPS + 1) * 32, smem, st>>>(c->ctx, out, seg_base, spw);
+  k_score<D, kScorePPS><<<grid, kScorePPS * 32, smem, st>>>(c->ctx, out, seg_base, nslots);
   FKV_LAUNCHED(c);
   return FKV_OK;
 }
@@ -391,20 +401,30 @@ int fkv_load_scorer(fkv_cache *c, int layer, int kv_head, const float *W1, const
   c->staging.assign(c->lay.sp_stride, 0);
   uint32_t *wkv = (uint32_t *)c->staging.data();
   auto w1 = [&](int row, int col) { return W1[(size_t)row * H + col]; };
-  auto pack = [&](int row, int col) {
-    return (uint32_t)f32_to_bf16_rne(w1(row, col)) | ((uint32_t)f32_to_bf16_rne(w1(row + 1, col)) << 16);
+  // Part 0 of a weight is its bf16 rounding, part 1 the bf16 rounding of what that left over.
+  auto part = [&](int row, int col, int which) {
+    const float w = w1(row, col);
+    const uint16_t hi = f32_to_bf16_rne(w);
+    if (which == 0) return hi;
+    if (!std::isfinite(bf16_to_f32(hi))) return (uint16_t)0;   // inf and NaN carry no remainder
+    return f32_to_bf16_rne(w - bf16_to_f32(hi));
+  };
+  auto pack = [&](int row, int col, int which) {
+    return (uint32_t)part(row, col, which) | ((uint32_t)part(row + 1, col, which) << 16);
   };
   // mma B fragments (16 x 8, "col"): lane (gid, tig) holds rows k0 + 2 tig (+1) and k0 + 8 + 2 tig (+1) of
-  // column gid; registers 0-1 for hidden units 0-7, 2-3 for hidden units 8-15.
-  for (int ks = 0; ks < KS; ++ks)
-    for (int lane = 0; lane < 32; ++lane) {
-      const int gid = lane >> 2, tig = lane & 3, k0 = ks * 16;
-      uint32_t *r = wkv + ((size_t)ks * 32 + lane) * 4;
-      r[0] = pack(k0 + 2 * tig, gid);
-      r[1] = pack(k0 + 8 + 2 * tig, gid);
-      r[2] = pack(k0 + 2 * tig, 8 + gid);
-      r[3] = pack(k0 + 8 + 2 * tig, 8 + gid);
-    }
+  // column gid; registers 0-1 for hidden units 0-7, 2-3 for hidden units 8-15.  All fragments of the
+  // roundings first, then all fragments of the remainders.
+  for (int which = 0; which < 2; ++which)
+    for (int ks = 0; ks < KS; ++ks)
+      for (int lane = 0; lane < 32; ++lane) {
+        const int gid = lane >> 2, tig = lane & 3, k0 = ks * 16;
+        uint32_t *r = wkv + ((size_t)(which * KS + ks) * 32 + lane) * 4;
+        r[0] = pack(k0 + 2 * tig, gid, which);
+        r[1] = pack(k0 + 8 + 2 * tig, gid, which);
+        r[2] = pack(k0 + 2 * tig, 8 + gid, which);
+        r[3] = pack(k0 + 8 + 2 * tig, 8 + gid, which);
+      }
   // Per quad lane t the hidden units {2t, 2t+1, 8+2t, 9+2t}: the mma accumulator columns that lane owns.
   auto quad = [&](float *dst, auto get) {
     for (int t = 0; t < 4; ++t) {
@@ -412,8 +432,35 @@ int fkv_load_scorer(fkv_cache *c, int layer, int kv_head, const float *W1, const
       dst[t * 4 + 2] = get(8 + 2 * t); dst[t * 4 + 3] = get(9 + 2 * t);
     }
   };
-  float *wf = (float *)(c->staging.data() + c->lay.sp_off_wf);
-  for (int f = 0; f < F; ++f) quad(wf + (size_t)f * 16, [&](int j) { return w1(2 * D + f, j); });
+  // Feature rows of W1 as tf32 mma B fragments (8 x 8, "col"): lane (gid, tig) holds rows k0 + tig and k0 + 4 + tig
+  // of column gid.  A weight is its truncation to tf32 (10 mantissa bits) plus the truncated remainder; per k-step
+  // and lane eight words: truncations for hidden units 0-7 and 8-15, then the remainders.  Rows past F are zero.
+  uint32_t *wf = (uint32_t *)(c->staging.data() + c->lay.sp_off_wf);
+  auto tf32_part = [&](int row, int col, int which) -> uint32_t {
+    if (row >= F) return 0u;
+    const float w = w1(2 * D + row, col);
+    uint32_t u;
+    memcpy(&u, &w, 4);
+    const uint32_t t = u & 0xffffe000u;
+    if (which == 0) return t;
+    float tf;
+    memcpy(&tf, &t, 4);
+    if (!std::isfinite(tf)) return 0u;
+    const float r = w - tf;
+    memcpy(&u, &r, 4);
+    return u & 0xffffe000u;
+  };
+  for (int ks = 0; ks < ScoreSmem::fk(F); ++ks)
+    for (int lane = 0; lane < 32; ++lane) {
+      const int gid = lane >> 2, tig = lane & 3, k0 = ks * 8;
+      uint32_t *r = wf + ((size_t)ks * 32 + lane) * 8;
+      for (int which = 0; which < 2; ++which) {
+        r[which * 4 + 0] = tf32_part(k0 + tig, gid, which);
+        r[which * 4 + 1] = tf32_part(k0 + 4 + tig, gid, which);
+        r[which * 4 + 2] = tf32_part(k0 + tig, 8 + gid, which);
+        r[which * 4 + 3] = tf32_part(k0 + 4 + tig, 8 + gid, which);
+      }
+    }
   quad((float *)(c->staging.data() + c->lay.sp_off_b1), [&](int j) { return b1[j]; });
   quad((float *)(c->staging.data() + c->lay.sp_off_w2), [&](int j) { return W2[j]; });
   *(float *)(c->staging.data() + c->lay.sp_off_b2) = b2;

@@ -3,20 +3,28 @@
 // streamed over every pair of the segments on the work list.
 //
 // Roofline: HBM.  A pair is 4D + 4F bytes in and 4 bytes out, but 2(2D+F)H
-// flops, which is more than the fp32 pipes can do at HBM speed, so the
-// [16 pairs x 2D] . [2D x 16] part runs as bf16 mma with fp32 accumulation;
-// the F feature columns stay in fp32 FMAs (they are not bf16 data).
+// flops, which is more than the fp32 pipes can do at HBM speed, so the whole
+// x W1 product runs on the tensor cores with fp32 accumulation and every
+// operand carried at (nearly) fp32 precision by splitting it into parts the
+// tensor cores multiply exactly:
+//   k, v (bf16 data) x W1 rows (fp32): bf16 mma, the weight as rounding +
+//       remainder (two bf16 values);
+//   a (fp32 data) x W1 rows (fp32): tf32 mma, feature and weight each as a
+//       truncation to tf32 + the remainder, three of the four cross products
+//       (the fourth is below 2^-20 of the term).
 //
 // Structure: persistent CTAs, one per SM, each a contiguous range of tiles
-// (NCW consecutive pages of one segment).  A producer warp brings whole page
-// records (16 pairs: K, V, features + positions, one contiguous block) from
-// HBM into shared memory with one bulk async copy per page.  Consumer warp w
-// takes page w of every tile and owns its own ring of page slots, each slot
-// with its own full/empty mbarrier pair, fed by lane w of the producer - the
-// warps never wait for one another.  ldmatrix reads the pre-swizzled K and V
-// rows as A fragments; the bf16 rows of W1 sit in registers as B fragments
-// and the fp32 feature rows in a per-warp shared-memory copy, both reloaded
-// when the segment (and so the scorer) changes.
+// (NCW consecutive pages of one segment).  The pages of the range go round a
+// ring of page slots in shared memory (as many as fit), each slot with its own
+// mbarrier, and round the warps: whole page records (16 pairs: K, V, features
+// + positions, one contiguous block) arrive from HBM by one bulk async copy
+// per page, issued into a slot by the warp that has just scored the slot's
+// previous page - no warp waits for another warp's progress, only for its own
+// page to land, and no warp is set aside for copying (eight warps, two per
+// scheduler, leave each thread 255 registers).  ldmatrix reads the pre-swizzled K and V rows as A fragments;
+// the K/V rows of W1 sit in registers as B fragments, the feature rows in a
+// per-warp shared-memory copy (also as B fragments).  Both are reloaded when
+// the segment (and so the scorer) changes.
 #pragma once
 #include "fkv_dev.cuh"
 
@@ -43,20 +51,44 @@ __device__ __forceinline__ int find_work(const int *start, int nwork, int t) {
 
 struct ScoreSmem {
   static __host__ __device__ int pitch(int page_bytes) { return (page_bytes + 127) & ~127; }
-  // slots [spw * ncw][pitch] | per-warp feature weights [ncw][F * 16 floats] | barriers
-  static __host__ __device__ size_t bytes(int page_bytes, int F, int ncw, int spw) {
-    return (size_t)spw * ncw * pitch(page_bytes) + (size_t)ncw * F * 64 + (size_t)spw * ncw * 16 + 128;
+  static __host__ __device__ int fk(int F) { return (F + 7) / 8; }   // 8-feature k-steps of the tf32 mma
+  // slots [nslots][pitch] | per-warp feature weights [ncw][fk][32 lanes][8 words] | barriers
+  static __host__ __device__ size_t bytes(int page_bytes, int F, int ncw, int nslots) {
+    return (size_t)nslots * pitch(page_bytes) + (size_t)ncw * fk(F) * 1024 + (size_t)nslots * 8 + 128;
   }
 };
 
+// The pages a CTA scores, in order: its tile range [t0, t1) of the plan's tile list covers, for every work item
+// (segment) it touches, a run of that segment's pages (the segment's last tile may be short).  v numbers the
+// pages of the whole range from 0; the walk only moves forward.
+struct PageWalk {
+  int wi, v0, cnt;   // current work item, the number of its first page in the range, its pages in the range
+  int p0, seg, n;    // that first page's index inside the segment, the segment, its length in pairs
+};
+__device__ __forceinline__ bool walk_to(const Ctx &c, PageWalk &w, int v, int t0, int t1, int nwork, int tile_pages) {
+  while (v >= w.v0 + w.cnt) {
+    w.v0 += w.cnt;
+    w.cnt = 0;
+    if (++w.wi >= nwork) return false;
+    const int tbeg = c.tile1_start[w.wi];
+    if (tbeg >= t1) return false;
+    const int tend = c.tile1_start[w.wi + 1];
+    w.seg = c.work[w.wi];
+    w.n = c.plan[w.seg].n_old;
+    w.p0 = (max(t0, tbeg) - tbeg) * tile_pages;
+    w.cnt = max(0, min((min(t1, tend) - tbeg) * tile_pages, (w.n + kPage - 1) / kPage) - w.p0);
+  }
+  return true;
+}
+
 // Scores of the two rows (gid, gid + 8) this lane holds a quarter of: bias, activation, W2 dot, quad reduction.
 template <int ACT>
-__device__ __forceinline__ void score_rows(const float (&acc)[2][4], const float (&fz)[2][4], const float4 &b1,
-                                           const float4 &w2, int act, float (&p)[2]) {
+__device__ __forceinline__ void score_rows(const float (&acc)[2][4], const float4 &b1, const float4 &w2, int act,
+                                           float (&p)[2]) {
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
-    const float z0 = acc[0][2 * r] + fz[r][0] + b1.x, z1 = acc[0][2 * r + 1] + fz[r][1] + b1.y;
-    const float z2 = acc[1][2 * r] + fz[r][2] + b1.z, z3 = acc[1][2 * r + 1] + fz[r][3] + b1.w;
+    const float z0 = acc[0][2 * r] + b1.x, z1 = acc[0][2 * r + 1] + b1.y;
+    const float z2 = acc[1][2 * r] + b1.z, z3 = acc[1][2 * r + 1] + b1.w;
     float q;
     if (ACT == 0)
       q = fmaxf(z0, 0.f) * w2.x + fmaxf(z1, 0.f) * w2.y + fmaxf(z2, 0.f) * w2.z + fmaxf(z3, 0.f) * w2.w;
@@ -68,19 +100,19 @@ __device__ __forceinline__ void score_rows(const float (&acc)[2][4], const float
   }
 }
 
-// out[(seg - seg_base) * cap + slot] receives the score of each pair.  spw = page slots per consumer warp.
+// out[(seg - seg_base) * cap + slot] receives the score of each pair.  nslots = page slots of the ring.
 template <int D, int NCW>
-__global__ void __launch_bounds__((NCW + 1) * 32, 1) k_score(Ctx c, float *out, int seg_base, int spw) {
+__global__ void __launch_bounds__(NCW * 32, 1) k_score(Ctx c, float *out, int seg_base, int nslots) {
   constexpr int KSH = D / 16;        // 16-channel k-steps per tensor (K, then V)
   extern __shared__ __align__(128) uint8_t smem[];
   const int pitch = ScoreSmem::pitch(c.page_bytes);
-  const int nslots = spw * NCW;
   float *wsm_all = reinterpret_cast<float *>(smem + (size_t)nslots * pitch);
-  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)nslots * pitch + (size_t)NCW * c.F * 64);  // full[], empty[]
+  const int FK = ScoreSmem::fk(c.F);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)nslots * pitch + (size_t)NCW * FK * 1024);  // full[]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 2 * nslots; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    for (int s = 0; s < nslots; ++s) mbar_init(smem_u32(&bars[s]), 1);
     fence_barrier_init();
   }
   __syncthreads();
@@ -89,141 +121,139 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) k_score(Ctx c, float *out, 
   const int per = (total + gridDim.x - 1) / gridDim.x;
   const int t0 = blockIdx.x * per, t1 = min(t0 + per, total);
   if (t0 >= t1) return;
-  constexpr int TILE = NCW * kPage;
-  int wi = find_work(c.tile1_start, nwork, t0);
-  // The work item a warp is in: its tiles [tbeg, tend), its segment and length.  Reloaded only on a change.
-  int tbeg = 0, tend = -1, seg = 0, n = 0;
+  const int wi0 = find_work(c.tile1_start, nwork, t0) - 1;
 
-  if (warp == NCW) {
-    // ---------------- producer: lane w feeds consumer warp w ----------------
-    if (lane >= NCW) return;
-    int ks = 0, ph = 0;   // this lane's next slot (of its spw) and the phase of that slot's barriers
-    auto lookup = [&](int t, int &pid) {   // page of tile t for this lane, or -1
-      if (t >= tend) {
-        while (t >= c.tile1_start[wi + 1]) ++wi;
-        tbeg = c.tile1_start[wi]; tend = c.tile1_start[wi + 1];
-        seg = c.work[wi];
-        n = c.plan[seg].n_old;
-      }
-      const int pg = (t - tbeg) * NCW + lane;
-      pid = pg * kPage < n ? c.pt[(size_t)seg * c.max_pages + pg] : -1;
-    };
-    const uint64_t stream_once = l2_policy_evict_first();   // every page passes through L2 exactly once here
-    int pid, pid_next = -1;
-    lookup(t0, pid);
-    for (int t = t0; t < t1; ++t) {
-      if (t + 1 < t1) lookup(t + 1, pid_next);   // in flight while this lane waits for its slot
-      if (pid >= 0) {
-        const int slot = lane + NCW * ks;
-        if (!mbar_wait(smem_u32(&bars[nslots + slot]), ph ^ 1)) { set_status(c, kDevWaitTimeout); break; }
-        mbar_arrive_expect_tx(smem_u32(&bars[slot]), (uint32_t)c.page_bytes);
-        bulk_g2s_hint(smem_u32(smem + (size_t)slot * pitch), c.pool + (size_t)pid * c.page_bytes,
-                      (uint32_t)c.page_bytes, smem_u32(&bars[slot]), stream_once);
-        if (++ks == spw) { ks = 0; ph ^= 1; }
-      }
-      pid = pid_next;
+  // Page v of the CTA's range lives in ring slot v % nslots and is scored by warp v % NCW; nslots is a multiple
+  // of NCW, so a slot always serves the same warp.  The warp that has finished with page v issues the copy of
+  // page v + nslots into the slot it has just freed (no "empty" barriers exist) and is the one to wait for it
+  // later: a slot's barrier is never more than one phase ahead of its only waiter.
+  PageWalk ahead = {wi0, 0, 0, 0, 0, 0};
+  const uint64_t stream_once = l2_policy_evict_first();   // every page passes through L2 exactly once here
+  auto fill = [&](int slot_i, int pid, uint32_t tie) {    // one bulk copy: the whole page record
+    if (lane == 0) {
+      const uint32_t bar = smem_u32(&bars[slot_i]);
+      fence_proxy_async();   // the reads of the slot's previous page come before the copy engine's writes
+      mbar_arrive_expect_tx(bar, (uint32_t)c.page_bytes);
+      bulk_g2s_hint(smem_u32(smem + (size_t)slot_i * pitch) + tie, c.pool + (size_t)pid * c.page_bytes,
+                    (uint32_t)c.page_bytes, bar, stream_once);
     }
-    return;
-  }
+  };
+  for (int v = warp; v < nslots; v += NCW)
+    if (walk_to(c, ahead, v, t0, t1, nwork, NCW))
+      fill(v, c.pt[(size_t)ahead.seg * c.max_pages + ahead.p0 + (v - ahead.v0)], 0u);
 
-  // ---------------- consumers: warp w owns page w of every tile ----------------
   const int gid = lane >> 2, tig = lane & 3;
-  uint32_t bw[2 * KSH][4];  // W1 (K rows, then V rows) as mma B fragments: both 8-wide halves of the 16 hidden units
-  float4 *wsm = reinterpret_cast<float4 *>(wsm_all + (size_t)warp * c.F * 16);   // feature rows of W1, [F][4 tig] float4
+  // W1 (K rows, then V rows) as mma B fragments, both 8-wide halves of the 16 hidden units.  An fp32 weight is
+  // carried as two bf16 values, its rounding (bw) and the rounding of what that left over (bl): the channels
+  // are bf16 already, so both products are exact and the weight enters with about 2^-17 relative error.
+  uint32_t bw[2 * KSH][4], bl[2 * KSH][4];
+  uint4 *wsm = reinterpret_cast<uint4 *>(wsm_all + (size_t)warp * FK * 256);   // feature rows of W1: [FK][lane] x 2 uint4
   float4 b1 = make_float4(0.f, 0.f, 0.f, 0.f), w2 = b1;
   float b2 = 0.f;
   // ldmatrix row address pieces for this lane: matrix mi = lane / 8 covers rows (mi & 1) * 8 .. +8
   // and the low (mi < 2) or high 8 channels of a 16-channel step.
   const int lrow = ((lane >> 3) & 1) * 8 + (lane & 7), lhi = lane >> 4;
-  int ks = 0, ph = 0;
   // The scores are read back by the selection kernel right away: keep them in L2, so that no write
   // goes to DRAM in the middle of the read stream.
   const uint64_t keep = l2_policy_evict_last();
 
-  for (int t = t0; t < t1; ++t) {
-    if (t >= tend) {
-      while (t >= c.tile1_start[wi + 1]) ++wi;
-      tbeg = c.tile1_start[wi]; tend = c.tile1_start[wi + 1];
-      seg = c.work[wi];
-      n = c.plan[seg].n_old;
-      const int spi = (seg / (c.batch * c.Hkv)) * c.Hkv + seg % c.Hkv;  // (layer, head)
+  PageWalk cur = {wi0, 0, 0, 0, 0, 0};
+  int scorer = -1;                   // (layer, head) whose weights the warp holds
+  int slot_i = warp, ph = 0;         // ring slot of page v and the parity of its barrier's current phase
+  for (int v = warp; walk_to(c, cur, v, t0, t1, nwork, NCW); v += NCW) {
+    // The page that will take this slot next: looked up now, copied when this page has been scored.
+    const int pid_next = walk_to(c, ahead, v + nslots, t0, t1, nwork, NCW)
+                             ? c.pt[(size_t)ahead.seg * c.max_pages + ahead.p0 + (v + nslots - ahead.v0)] : -1;
+    const int seg = cur.seg, n = cur.n, pg = cur.p0 + (v - cur.v0);
+    const int spi = (seg / (c.batch * c.Hkv)) * c.Hkv + seg % c.Hkv;  // (layer, head)
+    if (spi != scorer) {
+      scorer = spi;
       const uint8_t *sp = c.sp + (size_t)spi * c.sp_stride;
       const uint4 *w = reinterpret_cast<const uint4 *>(sp);
 #pragma unroll
       for (int k = 0; k < 2 * KSH; ++k) {
         uint4 x = __ldg(w + k * 32 + lane);
         bw[k][0] = x.x; bw[k][1] = x.y; bw[k][2] = x.z; bw[k][3] = x.w;
+        x = __ldg(w + (2 * KSH + k) * 32 + lane);
+        bl[k][0] = x.x; bl[k][1] = x.y; bl[k][2] = x.z; bl[k][3] = x.w;
       }
       __syncwarp();
-      const float4 *wf = reinterpret_cast<const float4 *>(sp + c.sp_off_wf);
-      for (int i = lane; i < c.F * 4; i += 32) wsm[i] = __ldg(wf + i);
+      const uint4 *wf = reinterpret_cast<const uint4 *>(sp + c.sp_off_wf);
+      for (int i = lane; i < FK * 64; i += 32) wsm[i] = __ldg(wf + i);
       b1 = __ldg(reinterpret_cast<const float4 *>(sp + c.sp_off_b1) + tig);
       w2 = __ldg(reinterpret_cast<const float4 *>(sp + c.sp_off_w2) + tig);
       b2 = __ldg(reinterpret_cast<const float *>(sp + c.sp_off_b2));
       __syncwarp();
     }
-    const int tin = t - tbeg;
-    if ((tin * NCW + warp) * kPage >= n) continue;   // the segment's last tile may have fewer pages
-    const int slot_i = warp + NCW * ks;
     if (!mbar_wait(smem_u32(&bars[slot_i]), ph)) { set_status(c, kDevWaitTimeout); break; }
     const uint8_t *page = smem + (size_t)slot_i * pitch;
     const uint32_t kbase = smem_u32(page), vbase = kbase + c.off_v;
-    // Four accumulation chains per half of the hidden units (K / V channels, even / odd k-steps),
-    // summed below in a fixed order: a quarter of the dependent-mma depth.
+    // Eight accumulators (four chains for each half of the hidden units), summed below in a fixed order, so that
+    // consecutive mma are independent.  The feature columns come first: x = xt + xr (truncation to tf32 and the
+    // remainder, both exact), w = wt + wr likewise (prepared by the host): xt wt + xr wt + xt wr.  This lane's
+    // part of the A fragment: rows gid and gid + 8, feature columns 8 ks + tig and + 4.
     float ac[4][2][4];
 #pragma unroll
     for (int q = 0; q < 4; ++q)
 #pragma unroll
       for (int h = 0; h < 2; ++h) ac[q][h][0] = ac[q][h][1] = ac[q][h][2] = ac[q][h][3] = 0.f;
+    const float *f0 = meta_row(c, page, gid), *f1 = meta_row(c, page, gid + 8);
+    for (int ks = 0; ks < FK; ++ks) {
+      const int c0 = ks * 8 + tig, c1 = c0 + 4;
+      float x[4];
+      x[0] = c0 < c.F ? f0[c0] : 0.f; x[1] = c0 < c.F ? f1[c0] : 0.f;   // past F sits the position id: never read as a feature
+      x[2] = c1 < c.F ? f0[c1] : 0.f; x[3] = c1 < c.F ? f1[c1] : 0.f;
+      uint32_t xt[4], xr[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        xt[i] = __float_as_uint(x[i]) & 0xffffe000u;
+        xr[i] = __float_as_uint(x[i] - __uint_as_float(xt[i])) & 0xffffe000u;
+      }
+      const uint4 wt = wsm[(ks * 32 + lane) * 2], wr = wsm[(ks * 32 + lane) * 2 + 1];
+      mma_tf32(ac[0][0], xt[0], xt[1], xt[2], xt[3], wt.x, wt.y);
+      mma_tf32(ac[0][1], xt[0], xt[1], xt[2], xt[3], wt.z, wt.w);
+      mma_tf32(ac[1][0], xr[0], xr[1], xr[2], xr[3], wt.x, wt.y);
+      mma_tf32(ac[1][1], xr[0], xr[1], xr[2], xr[3], wt.z, wt.w);
+      mma_tf32(ac[2][0], xt[0], xt[1], xt[2], xt[3], wr.x, wr.y);
+      mma_tf32(ac[2][1], xt[0], xt[1], xt[2], xt[3], wr.z, wr.w);
+    }
+    // K (chains 0: roundings, 1: remainders of the weights) and V (chains 2, 3).
 #pragma unroll
     for (int kk = 0; kk < KSH; ++kk) {           // 16-channel step inside K and inside V
       const int ch = kk * 2 + lhi;               // 16-byte chunk this lane addresses
       uint32_t a[4], b[4];
       ldsm_x4(a, kbase + kv_chunk_off(lrow, ch, D));
       ldsm_x4(b, vbase + kv_chunk_off(lrow, ch, D));
-      mma_bf16(ac[kk & 1][0], a[0], a[1], a[2], a[3], bw[kk][0], bw[kk][1]);
-      mma_bf16(ac[kk & 1][1], a[0], a[1], a[2], a[3], bw[kk][2], bw[kk][3]);
-      mma_bf16(ac[2 + (kk & 1)][0], b[0], b[1], b[2], b[3], bw[KSH + kk][0], bw[KSH + kk][1]);
-      mma_bf16(ac[2 + (kk & 1)][1], b[0], b[1], b[2], b[3], bw[KSH + kk][2], bw[KSH + kk][3]);
+      mma_bf16(ac[0][0], a[0], a[1], a[2], a[3], bw[kk][0], bw[kk][1]);
+      mma_bf16(ac[0][1], a[0], a[1], a[2], a[3], bw[kk][2], bw[kk][3]);
+      mma_bf16(ac[2][0], b[0], b[1], b[2], b[3], bw[KSH + kk][0], bw[KSH + kk][1]);
+      mma_bf16(ac[2][1], b[0], b[1], b[2], b[3], bw[KSH + kk][2], bw[KSH + kk][3]);
+      mma_bf16(ac[1][0], a[0], a[1], a[2], a[3], bl[kk][0], bl[kk][1]);
+      mma_bf16(ac[1][1], a[0], a[1], a[2], a[3], bl[kk][2], bl[kk][3]);
+      mma_bf16(ac[3][0], b[0], b[1], b[2], b[3], bl[KSH + kk][0], bl[KSH + kk][1]);
+      mma_bf16(ac[3][1], b[0], b[1], b[2], b[3], bl[KSH + kk][2], bl[KSH + kk][3]);
     }
     float acc[2][4];
 #pragma unroll
     for (int h = 0; h < 2; ++h)
 #pragma unroll
       for (int i = 0; i < 4; ++i) acc[h][i] = (ac[0][h][i] + ac[1][h][i]) + (ac[2][h][i] + ac[3][h][i]);
-    // Feature columns in fp32: this lane owns hidden units {2t, 2t+1, 8+2t, 9+2t} of rows gid and gid+8.
-    float fz[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-    const float *f0 = meta_row(c, page, gid), *f1 = meta_row(c, page, gid + 8);   // odd word stride: no bank conflicts
-    for (int f = 0; f < c.F; f += 6) {   // one query head's six features at a time: all loads, then the FMAs
-      float x0[6], x1[6];
-      float4 w[6];
-#pragma unroll
-      for (int j = 0; j < 6; ++j) {
-        x0[j] = f0[f + j]; x1[j] = f1[f + j];
-        w[j] = wsm[(f + j) * 4 + tig];
-      }
-#pragma unroll
-      for (int j = 0; j < 6; ++j) {
-        fz[0][0] = fmaf(x0[j], w[j].x, fz[0][0]); fz[0][1] = fmaf(x0[j], w[j].y, fz[0][1]);
-        fz[0][2] = fmaf(x0[j], w[j].z, fz[0][2]); fz[0][3] = fmaf(x0[j], w[j].w, fz[0][3]);
-        fz[1][0] = fmaf(x1[j], w[j].x, fz[1][0]); fz[1][1] = fmaf(x1[j], w[j].y, fz[1][1]);
-        fz[1][2] = fmaf(x1[j], w[j].z, fz[1][2]); fz[1][3] = fmaf(x1[j], w[j].w, fz[1][3]);
-      }
-    }
     float p[2];
-    if (c.act == 0) score_rows<0>(acc, fz, b1, w2, 0, p);
-    else score_rows<1>(acc, fz, b1, w2, c.act, p);
+    if (c.act == 0) score_rows<0>(acc, b1, w2, 0, p);
+    else score_rows<1>(acc, b1, w2, c.act, p);
     // Every lane of a quad holds both sums; lane l < 16 takes the score of row l (from quad l % 8), so
     // the page's sixteen scores leave as one 64-byte store.
     const float lo = __shfl_sync(0xffffffffu, p[0], (lane & 7) * 4), hi = __shfl_sync(0xffffffffu, p[1], (lane & 7) * 4);
     const float mine = lane < 8 ? lo : hi;
-    const int slot = tin * TILE + warp * kPage + lane;
+    const int slot = pg * kPage + lane;
     if (lane < kPage && slot < n) st_f32_hint(out + (size_t)(seg - seg_base) * c.cap + slot, mine + b2, keep);
-    // The slot may be refilled as soon as this arrival is seen: tie it to the score, which depends on every value
-    // read from the page, through a zero the compiler cannot see through (the grid is one-dimensional).
+    // The slot is refilled at once, and must not be before every read of the page has returned: tie the copy's
+    // destination to the score, which depends on every value read from the page, through a zero the
+    // compiler cannot see through (the grid is one-dimensional).
     __syncwarp();
-    if (lane == 0) mbar_arrive(smem_u32(&bars[nslots + slot_i]) + (__float_as_uint(mine) & (gridDim.y - 1)));
-    if (++ks == spw) { ks = 0; ph ^= 1; }
+    if (pid_next >= 0) fill(slot_i, pid_next, __float_as_uint(mine) & (gridDim.y - 1));
+    slot_i += NCW;
+    if (slot_i >= nslots) { slot_i -= nslots; ph ^= 1; }
   }
 }
 

@@ -117,9 +117,8 @@ def shrink(w: Workload, num_layers: int | None = None, max_len: int | None = Non
 def scorer_params(w: Workload, layer: int, device="cpu"):
     """Random-init scorer of one layer: W1 [Hkv][2D+6g][H], b1 [Hkv][H], W2 [Hkv][H], b2 [Hkv], fp32.
 
-    U(-1/sqrt(fan_in), +1/sqrt(fan_in)).  The K and V rows of W1 are made
-    representable in bf16 (the model and its cache are bf16), so a library that
-    stores those rows as bf16 loses nothing.
+    U(-1/sqrt(fan_in), +1/sqrt(fan_in)), plain fp32 as a trainer would hand
+    them over.
     """
     g = _gen(w, device, _T_W, layer)
     Hk, X, H = w.num_kv_heads, w.x_dim, w.scorer_hidden
@@ -128,7 +127,6 @@ def scorer_params(w: Workload, layer: int, device="cpu"):
     b1 = (torch.rand((Hk, H), generator=g, device=device) * 2 - 1) * b_in
     W2 = (torch.rand((Hk, H), generator=g, device=device) * 2 - 1) * b_hid
     b2 = (torch.rand((Hk,), generator=g, device=device) * 2 - 1) * b_hid
-    W1[:, : 2 * w.head_dim, :] = W1[:, : 2 * w.head_dim, :].to(torch.bfloat16).to(torch.float32)
     return W1.contiguous(), b1.contiguous(), W2.contiguous(), b2.contiguous()
 
 

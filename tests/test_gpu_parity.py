@@ -21,6 +21,9 @@ from util import bits, bits_to_f64, npf
 pytestmark = pytest.mark.gpu
 
 SCORE_TOL = 1e-3
+# N(0,1) inputs and fp32 weights below 0.1: sums of about 2D products of magnitude <= 0.3 accumulated in fp32
+# (2^-24 relative per step), weights carried to 2^-17 relative: errors of a few 1e-6.
+SCORE_TOL_FP32_WEIGHTS = 3e-5
 ATTN_TOL = 2e-2
 
 
@@ -100,6 +103,54 @@ def test_score_other_activations(act):
         K, V, A, _ = ld.head(0, 0, h)
         ref = oracle.score(K, V, A, *ld.weights(0, h), act=act)
         assert np.abs(got[0, h, :w.lens[0]] - ref).max() <= SCORE_TOL
+
+
+def _score_with_weights(w, W1, b1, W2, b2):
+    """Scores of config-1 data under the given scorer of every head: (GPU fp32, oracle fp32)."""
+    ld = Loaded(w)
+    for h in range(w.num_kv_heads):
+        ld.cache.load_scorer(0, h, torch.from_numpy(W1[h]), torch.from_numpy(b1[h]), torch.from_numpy(W2[h]), float(b2[h]))
+    got = npf(ld.cache.score(0))
+    ref = np.stack([oracle.score(*ld.head(0, 0, h)[:3], W1[h], b1[h], W2[h], float(b2[h])) for h in range(w.num_kv_heads)])
+    assert ld.cache.device_status()[0] == 0
+    return got[0, :, :w.lens[0]], ref, ld
+
+
+def test_score_weights_half_way_between_bf16_values():
+    # Appendix B.1 gives W1 no precision, so weights arrive as fp32.  Here every K/V weight lies EXACTLY half-way
+    # between two neighbouring bf16 values (17 significant bits): stored as a single bf16 it would be off by
+    # 2^-9 relative whichever way it is rounded, and the scores by ~1e-3; stored as rounding + remainder it is
+    # exact, and what is left is fp32 accumulation (~1e-6).  A dropped, mis-signed or truncated remainder fails.
+    w = small(1)
+    rng = np.random.default_rng(5)
+    Hk, X, H, D = w.num_kv_heads, w.x_dim, w.scorer_hidden, w.head_dim
+    W1 = rng.uniform(-1, 1, (Hk, X, H)).astype(np.float32) / np.float32(np.sqrt(X))
+    kv = W1[:, :2 * D].view(np.uint32)
+    W1[:, :2 * D] = ((kv & np.uint32(0xFFFF0000)) | np.uint32(0x8000)).view(np.float32)
+    b1 = rng.uniform(-0.1, 0.1, (Hk, H)).astype(np.float32)
+    W2 = rng.uniform(-0.25, 0.25, (Hk, H)).astype(np.float32)
+    b2 = rng.uniform(-0.25, 0.25, Hk).astype(np.float32)
+    got, ref, ld = _score_with_weights(w, W1, b1, W2, b2)
+    assert np.abs(got - ref).max() <= SCORE_TOL_FP32_WEIGHTS, np.abs(got - ref).max()
+    # the same weights rounded to ONE bf16 value (to nearest even) must be measurably worse in the oracle itself,
+    # or the case would prove nothing
+    W1r = W1.copy()
+    W1r[:, :2 * D] = torch.from_numpy(W1[:, :2 * D].copy()).to(torch.bfloat16).float().numpy()
+    worse = np.stack([oracle.score(*ld.head(0, 0, h)[:3], W1r[h], b1[h], W2[h], float(b2[h])) for h in range(Hk)])
+    assert np.abs(worse - ref).max() > 10 * SCORE_TOL_FP32_WEIGHTS
+
+
+def test_score_plain_fp32_weights_tight():
+    # Unrounded U(+-1/sqrt(fan_in)) weights, as a trainer hands them over: far inside 1e-3.
+    w = small(1)
+    ld = Loaded(w)
+    got = npf(ld.cache.score(0))
+    for h in range(w.num_kv_heads):
+        K, V, A, _ = ld.head(0, 0, h)
+        W1 = ld.weights(0, h)[0]
+        assert np.any(torch.from_numpy(W1[:2 * w.head_dim].copy()).to(torch.bfloat16).float().numpy() != W1[:2 * w.head_dim])
+        ref = oracle.score(K, V, A, *ld.weights(0, h))
+        assert np.abs(got[0, h, :w.lens[0]] - ref).max() <= SCORE_TOL_FP32_WEIGHTS
 
 
 def test_score_duplicates_tie_bit_for_bit():
