@@ -119,11 +119,17 @@ int fkv_reset(fkv_cache *c, void *stream);
 int fkv_load_scorer(fkv_cache *c, int layer, int kv_head, const float *W1, const float *b1, const float *W2, float b2,
                     void *stream);
 
-/* Per-sequence budget B (host value; takes effect for later fkv_evict calls). */
+/*
+ * Per-sequence budget B - Section 3.1 states the problem with one budget B per cache; the batched
+ * configurations give every sequence its own (B = half its context), so the budget is a property of
+ * the sequence.  Host value; takes effect for later fkv_evict calls.
+ */
 int fkv_set_budget(fkv_cache *c, int seq, int32_t budget, void *stream);
 
 /*
- * Bulk-load one EMPTY (layer, sequence): n pairs per KV head.
+ * Bulk-load one EMPTY (layer, sequence): n pairs per KV head - the cache as the prefill phase leaves
+ * it (Section 3.1 starts from a cache that already holds the prompt; the one-shot compression mode of
+ * Section 4.4 evicts right after this call).  The paper has no counterpart for the call itself.
  * k, v: dev [Hkv][n][D] bf16; feat: dev [Hkv][n][F] fp32 or NULL (zeros);
  * pos: dev [n] int32 (strictly increasing token positions) or NULL (0..n-1).
  */
@@ -140,7 +146,12 @@ int fkv_prefill(fkv_cache *c, int layer, int seq, const void *k, const void *v, 
 int fkv_append(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, uint64_t seq_mask,
                void *stream);
 
-/* Overwrite the feature rows of one (layer, sequence): feat dev [Hkv][n][F] fp32, n = current length. */
+/*
+ * Overwrite the attention features a_n (Appendix B.1: six per query head and pair) of one (layer,
+ * sequence) with values computed elsewhere: feat dev [Hkv][n][F] fp32, n = current length.  For
+ * callers that maintain the features themselves (feature_window = 0) and for checks; the paper has no
+ * counterpart for the call itself.
+ */
 int fkv_set_features(fkv_cache *c, int layer, int seq, const float *feat, void *stream);
 
 /*
@@ -235,12 +246,18 @@ int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *p
 
 /* ---- staged entry points: one kernel each, for per-step checks ---- */
 
-/* Scores of every pair of `layer`: scores_out dev [max_batch][Hkv][cap] fp32, cap = fkv_score_stride. */
+/*
+ * The scorer alone - Appendix B.1: phi_n = sigma(Concat(k_n, v_n, a_n) W1 + b1) W2 + b2 for every pair
+ * of `layer`, with the (layer, KV head)'s own weights (Section 3.1: one scoring model per layer and
+ * attention group).  scores_out dev [max_batch][Hkv][cap] fp32, cap = fkv_score_stride.
+ */
 int fkv_score(fkv_cache *c, int layer, float *scores_out, void *stream);
 /*
- * Selection from given scores (dev, same layout): writes for each segment the
- * kept slots, ascending, to idx_out dev [max_batch][Hkv][cap] int32 and their
- * number min(B, n) to kept_count_out dev [max_batch][Hkv].
+ * The selection alone - Section 3.1: the most recent R pairs stay, the others are pruned back to
+ * B - R by score (the lowest scores are evicted; the Top-K row of the paper's sampling ablation, i.e.
+ * the deterministic action; ties: higher score, then lower slot).  From given scores (dev, layout as
+ * fkv_score writes them) writes for each segment the kept slots, ascending, to idx_out dev
+ * [max_batch][Hkv][cap] int32 and their number min(B, n) to kept_count_out dev [max_batch][Hkv].
  */
 int fkv_select(fkv_cache *c, int layer, const float *scores_in, int32_t *idx_out, int32_t *kept_count_out,
                void *stream);
@@ -248,9 +265,10 @@ int fkv_select(fkv_cache *c, int layer, const float *scores_in, int32_t *idx_out
 int fkv_select_sampled(fkv_cache *c, int layer, const float *scores_in, const float *noise, int32_t noise_stride,
                        int32_t *idx_out, int32_t *kept_count_out, void *stream);
 /*
- * Compaction by given ascending slot lists (dev, layout as fkv_select writes
- * them; every (sequence) must have the same count on all its heads).
- * Syncs (reads the new lengths back).
+ * The compaction alone - Section 3.1's state update s' = s \ D: the kept pairs' K, V, feature and
+ * position rows move, in order, into fresh pages and the segment's length becomes the kept count.
+ * By given ascending slot lists (dev, layout as fkv_select writes them; every sequence must have the
+ * same count on all its heads).  Syncs (reads the new lengths back).
  */
 int fkv_compact(fkv_cache *c, int layer, const int32_t *idx, const int32_t *kept_count, void *stream);
 
@@ -276,14 +294,22 @@ int fkv_update_features(fkv_cache *c, int layer, void *stream);
 /* Row stride, in elements, of the score and index arrays above. */
 int fkv_score_stride(const fkv_cache *c, int32_t *cap);
 
-/* Dense copy of one segment: k, v dev [n][D] bf16, feat dev [n][F], pos dev [n]; any may be NULL. */
+/*
+ * Dense copy of one segment: k, v dev [n][D] bf16, feat dev [n][F], pos dev [n]; any may be NULL.
+ * The paper has no counterpart: a read-out for checks and for moving a cache elsewhere.
+ */
 int fkv_export_head(fkv_cache *c, int layer, int seq, int kv_head, void *k, void *v, float *feat, int32_t *pos,
                     void *stream);
 
 /* Current lengths of `layer`: host_out [max_batch] (host mirror, no device access). */
 int fkv_get_lengths(const fkv_cache *c, int layer, int32_t *host_out);
 
-/* Reads the device status word and free-page count (syncs `stream`); clears the word. */
+/*
+ * Reads the device status word and free-page count (syncs `stream`); clears the word.
+ * When it returns FKV_ERR_DEVICE, a kernel has skipped work the host had already counted (an append, or
+ * a whole eviction step), so the host's copy of the lengths may be ahead of the device: call
+ * fkv_sync_lengths (or fkv_reset) before any other call on this handle.
+ */
 int fkv_device_status(fkv_cache *c, uint32_t *status_bits, int32_t *free_pages, void *stream);
 
 /*
@@ -323,6 +349,10 @@ int fkv_launch_count(const fkv_cache *c, uint64_t *launches);
  * [num_kv_heads][n][head_dim] bf16, dense row-major; scale 0 means
  * 1/sqrt(head_dim).  Same arithmetic as fkv_decode_attn (fp32 online softmax,
  * bf16 result), for one sequence.
+ *
+ * k and v must be 8-byte aligned (FKV_ERR_INVALID_ARG otherwise).  This is a
+ * service path: it reads one row per warp and step and is far slower than
+ * fkv_decode_attn for long sequences.
  *
  * Limits: head_dim 64 or 128 (else FKV_ERR_INVALID_ARG); 1 <= n <=
  * FKV_NOALLOC_MAX_PAIRS, num_kv_heads <= FKV_NOALLOC_MAX_KV_HEADS, group_size

@@ -151,6 +151,11 @@ struct fkv_cache {
   cudaEvent_t ev[7] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};  // [6]: after the plan
 };
 
+namespace fkv {
+// For the library's other translation units: record the text of a failed CUDA call for fkv_last_cuda_error.
+void note_cuda_error(cudaError_t e) { g_cuda_error = cudaGetErrorString(e); }
+}  // namespace fkv
+
 namespace {
 
 int cuda_fail(cudaError_t e) {

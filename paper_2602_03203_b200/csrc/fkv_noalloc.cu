@@ -22,6 +22,10 @@
 
 #include "../../include/fkv.h"
 
+namespace fkv {
+void note_cuda_error(cudaError_t e);   // fkv_api.cu: keeps the text fkv_last_cuda_error returns
+}
+
 namespace fkv_noalloc {
 
 constexpr int kMaxHeads = 16;    // KV heads per call
@@ -43,7 +47,23 @@ __device__ __forceinline__ float warp_sum(float x) {
   return x;
 }
 
-// grid (splits, Hkv), 128 threads.  CPL = channels per lane = D / 32.
+// CPL consecutive bf16 channels (CPL * 2 bytes, aligned to that) as floats.
+template <int CPL>
+__device__ __forceinline__ void load_channels(const __nv_bfloat16 *p, float (&x)[CPL]) {
+  static_assert(CPL == 2 || CPL == 4, "head_dim 64 or 128");
+  if (CPL == 2) {
+    const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(p));
+    x[0] = f.x; x[1] = f.y;
+  } else {
+    const uint2 u = *reinterpret_cast<const uint2 *>(p);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u.y));
+    x[0] = a.x; x[1] = a.y; x[CPL - 2] = b.x; x[CPL - 1] = b.y;
+  }
+}
+
+// grid (splits, Hkv), 128 threads.  CPL = channels per lane = D / 32.  A service path, not a tuned one: a warp
+// reads one row per step (256 bytes), far below the paged kernel's rate for long sequences.
 template <int CPL>
 __global__ void __launch_bounds__(128) k_attend_dense(const __nv_bfloat16 *q, const __nv_bfloat16 *k,
                                                       const __nv_bfloat16 *v, int n, int G, float scale_log2,
@@ -69,11 +89,8 @@ __global__ void __launch_bounds__(128) k_attend_dense(const __nv_bfloat16 *q, co
   }
   for (int i = i0 + warp; i < i1; i += 4) {
     float kr[CPL], vr[CPL];
-#pragma unroll
-    for (int c = 0; c < CPL; ++c) {
-      kr[c] = __bfloat162float(kh[(size_t)i * D + lane * CPL + c]);
-      vr[c] = __bfloat162float(vh[(size_t)i * D + lane * CPL + c]);
-    }
+    load_channels<CPL>(kh + (size_t)i * D + lane * CPL, kr);   // one 4- or 8-byte load per lane and tensor
+    load_channels<CPL>(vh + (size_t)i * D + lane * CPL, vr);
 #pragma unroll
     for (int h = 0; h < kMaxG; ++h) {
       if (h >= G) break;
@@ -168,13 +185,21 @@ extern "C" int fkv_decode_attn_dense_noalloc(const void *q, const void *k, const
   if (num_kv_heads < 1 || num_kv_heads > FKV_NOALLOC_MAX_KV_HEADS) return FKV_ERR_CAPACITY;
   if (group_size < 1 || group_size > kMaxG) return FKV_ERR_CAPACITY;
   static_assert(FKV_NOALLOC_MAX_KV_HEADS == kMaxHeads, "header and kernel disagree");
+  // k and v are read with one 8-byte (head_dim 128) or 4-byte (64) load per lane.
+  if ((((uintptr_t)k | (uintptr_t)v) & 7u) != 0) return FKV_ERR_INVALID_ARG;
+  auto failed = [](cudaError_t e) {
+    fkv::note_cuda_error(e);
+    return (int)FKV_ERR_CUDA;
+  };
   void *base = nullptr;
-  if (scratch_address(&base) != cudaSuccess) return FKV_ERR_CUDA;
+  cudaError_t err = scratch_address(&base);
+  if (err != cudaSuccess) return failed(err);
   float *part = (float *)base;
   int *tickets = (int *)((unsigned char *)base + kPartFloats * sizeof(float));
   cudaStream_t st = (cudaStream_t)stream;
   // The array keeps whatever the last call left; only the tickets must start at zero.
-  if (cudaMemsetAsync(tickets, 0, kMaxHeads * sizeof(int), st) != cudaSuccess) return FKV_ERR_CUDA;
+  err = cudaMemsetAsync(tickets, 0, kMaxHeads * sizeof(int), st);
+  if (err != cudaSuccess) return failed(err);
   int splits = (n + 255) / 256;
   splits = splits < 1 ? 1 : (splits > kMaxSplits ? kMaxSplits : splits);
   if (scale == 0.f) scale = 1.f / sqrtf((float)head_dim);
@@ -188,5 +213,6 @@ extern "C" int fkv_decode_attn_dense_noalloc(const void *q, const void *k, const
     k_attend_dense<2><<<grid, 128, 0, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                                             (const __nv_bfloat16 *)v, n, group_size, scale_log2, (__nv_bfloat16 *)out,
                                             part, tickets);
-  return cudaGetLastError() == cudaSuccess ? FKV_OK : FKV_ERR_CUDA;
+  err = cudaGetLastError();
+  return err == cudaSuccess ? (int)FKV_OK : failed(err);
 }

@@ -158,15 +158,17 @@ __global__ void __launch_bounds__(NCW * 32, 1) k_score(Ctx c, float *out, int se
   const uint64_t keep = l2_policy_evict_last();
 
   PageWalk cur = {wi0, 0, 0, 0, 0, 0};
-  int scorer = -1;                   // (layer, head) whose weights the warp holds
+  int scorer = -1, seg_held = -1;    // (layer, head) whose weights the warp holds; the segment last seen
   int slot_i = warp, ph = 0;         // ring slot of page v and the parity of its barrier's current phase
   for (int v = warp; walk_to(c, cur, v, t0, t1, nwork, NCW); v += NCW) {
     // The page that will take this slot next: looked up now, copied when this page has been scored.
     const int pid_next = walk_to(c, ahead, v + nslots, t0, t1, nwork, NCW)
                              ? c.pt[(size_t)ahead.seg * c.max_pages + ahead.p0 + (v + nslots - ahead.v0)] : -1;
     const int seg = cur.seg, n = cur.n, pg = cur.p0 + (v - cur.v0);
-    const int spi = (seg / (c.batch * c.Hkv)) * c.Hkv + seg % c.Hkv;  // (layer, head)
-    if (spi != scorer) {
+    if (seg != seg_held) {           // the divisions below only when the segment changes
+      seg_held = seg;
+      const int spi = (seg / (c.batch * c.Hkv)) * c.Hkv + seg % c.Hkv;  // (layer, head)
+      if (spi != scorer) {
       scorer = spi;
       const uint8_t *sp = c.sp + (size_t)spi * c.sp_stride;
       const uint4 *w = reinterpret_cast<const uint4 *>(sp);
@@ -184,6 +186,7 @@ __global__ void __launch_bounds__(NCW * 32, 1) k_score(Ctx c, float *out, int se
       w2 = __ldg(reinterpret_cast<const float4 *>(sp + c.sp_off_w2) + tig);
       b2 = __ldg(reinterpret_cast<const float *>(sp + c.sp_off_b2));
       __syncwarp();
+      }
     }
     if (!mbar_wait(smem_u32(&bars[slot_i]), ph)) { set_status(c, kDevWaitTimeout); break; }
     const uint8_t *page = smem + (size_t)slot_i * pitch;
