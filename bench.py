@@ -3,13 +3,15 @@
 
 A step is one pass of the whole hot path over one batch of synthetic input:
 one budgeted eviction over all layers (score -> select -> compact), then T
-decode tokens (append + GQA decode attention in every layer).  The cache is
-put back to its pre-eviction content between steps (untimed), and an L2-sized
-buffer is overwritten so every step starts cold.
+decode tokens, each one launch per layer of append + GQA decode attention (the
+per-layer call a model with projections between its layers makes).  The cache
+is put back to its pre-eviction content between steps (untimed), and an
+L2-sized buffer is overwritten so every step starts cold.
 
 Prints ONE JSON line.  `value` is the eviction step's algorithmic HBM
 throughput (GB/s); decode tokens/s, per-kernel times, the roofline of the
-dominant kernel and the CPU oracle's timing ride along.
+dominant kernel, the budget sweep of the 32K configuration and the CPU
+oracle's timing ride along.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                   [--config 1..5] [--budget B] [--decode-tokens T]
@@ -63,6 +65,21 @@ def evict_bytes(w, num_layers):
 
 def decode_bytes_per_token(w, num_layers, lens_now):
     return sum(num_layers * w.num_kv_heads * n * 4 * w.head_dim for n in lens_now)
+
+
+def profiled_traffic(kernel, units, budget):
+    """DRAM bytes per launch of `kernel` from its ncu capture: profiles/traffic.json holds the measured
+    bytes per unit (scored pair, kept pair at a budget), written beside the capture's summary; the
+    launch's traffic is that times its units (traffic is proportional to them).  None when the file
+    has no figure for this kernel (e.g. the kernel changed since its counters were taken)."""
+    try:
+        t = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))[kernel]
+    except Exception:
+        return None
+    per = t.get("bytes_per_unit")
+    if isinstance(per, dict):
+        per = per.get(str(budget))
+    return per * units if per else None
 
 
 def measured_peak():
@@ -205,7 +222,14 @@ def run_ours(args):
     if chunk_mode:
         T = args.decode_tokens = w.recent_keep if args.decode_tokens == 16 else args.decode_tokens
         w = dataclasses.replace(w, lens=tuple(min(n, b) for n, b in zip(w.lens, w.budgets)))
-    cache = binding.from_workload(w, L, max_tokens=max(w.lens) + max(256, T), feature_window=args.feature_window)
+    # The default run of the 32K configuration also times the eviction at the other two budgets of its sweep:
+    # the pool gets the fresh pages of the largest one.
+    sweep = [b for b in (2048, 8192, 16384) if b != max(w.budgets)] if (args.config == 3 and args.budget is None
+                                                                        and not args.no_sweep) else []
+    w_cap = dataclasses.replace(w, budgets=tuple(max([b] + sweep) for b in w.budgets))
+    cache = binding.from_workload(w_cap, L, max_tokens=max(w.lens) + max(256, T), feature_window=args.feature_window)
+    for s_, b in enumerate(w.budgets):
+        cache.set_budget(s_, b)
     for l in range(L):
         cache.load_scorers(l, *wl.scorer_params(w, l, dev))
         for s in range(w.batch):
@@ -235,6 +259,8 @@ def run_ours(args):
     cache.set_timing(True)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
 
+    views = [[(kd[t][l], vd[t][l], qd[t][l], od[t][l]) for l in range(L)] for t in range(T)]
+
     def one_step(e2e: bool):
         cache.restore(snap)
         flush.fill_(1)
@@ -245,7 +271,9 @@ def run_ours(args):
         ev[1].record()
         if chunk_mode:
             for t in range(T):
-                cache.decode_step(kd[t], vd[t], qd[t], od[t])
+                for l in range(L):
+                    k_, v_, q_, o_ = views[t][l]
+                    cache.append_decode_attn(l, k_, v_, q_, o_)
             ev[2].record()
             cache.evict(binding.ALL_LAYERS)
             if e2e:
@@ -257,7 +285,9 @@ def run_ours(args):
         cache.evict(binding.ALL_LAYERS)
         ev[2].record()
         for t in range(T):
-            cache.decode_step(kd[t], vd[t], qd[t], od[t])
+            for l in range(L):
+                k_, v_, q_, o_ = views[t][l]
+                cache.append_decode_attn(l, k_, v_, q_, o_)
         if e2e:
             oh.copy_(od, non_blocking=True)
         ev[3].record()
@@ -291,25 +321,22 @@ def run_ours(args):
         ev[0].record(); cache.evict_sampled(noise); ev[1].record(); torch.cuda.synchronize()
         sampled_ms.append(ev[0].elapsed_time(ev[1]))
     sampled_ms = ranks.max(min(sampled_ms[1:]))
-    # The same decode tokens with one ordinary launch per layer (fkv_append_decode_attn), i.e. without letting the
-    # layers of a token overlap: what a model sees whose projections sit between the layers.
-    serial_ms = 0.0
+    # The same decode tokens through fkv_decode_step, which is given every layer's k / v / q up front and lets the
+    # launches of consecutive layers overlap: a figure for engines that have them (and for the attention side
+    # alone), not what a model with projections between its layers can have.
+    over_ms = 0.0
     if T:
-        Ts = min(T, 4)
-        views = [[(kd[t][l], vd[t][l], qd[t][l], od[t][l]) for l in range(L)] for t in range(Ts)]
-        serial = []
+        over = []
         for _ in range(3):
             cache.restore(snap); torch.cuda.synchronize()
             if not chunk_mode:
                 cache.evict(); torch.cuda.synchronize()
             ev[0].record()
-            for t in range(Ts):
-                for l in range(L):
-                    k_, v_, q_, o_ = views[t][l]
-                    cache.append_decode_attn(l, k_, v_, q_, o_)
+            for t in range(T):
+                cache.decode_step(kd[t], vd[t], qd[t], od[t])
             ev[1].record(); torch.cuda.synchronize()
-            serial.append(ev[0].elapsed_time(ev[1]) / (Ts * L))
-        serial_ms = ranks.max(min(serial[1:]))
+            over.append(ev[0].elapsed_time(ev[1]) / (T * L))
+        over_ms = ranks.max(min(over[1:]))
     # The decode step recorded once into a CUDA graph and replayed per token (fixed k / v / q buffers): the host
     # launches one graph instead of one kernel per layer, which matters where the step is launch-bound.
     graph_ms = 0.0
@@ -336,10 +363,37 @@ def run_ours(args):
             reps.append(ev[0].elapsed_time(ev[1]) / (T * L))
         cache.sync_lengths()
         graph_ms = ranks.max(min(reps[1:]))
+    # Budget sweep of the 32K configuration: the same all-layer eviction at the other budgets (cache restored and
+    # L2 overwritten before each repetition, as in the timed steps).
+    mean = lambda xs: sum(xs) / len(xs)
+    peak, peak_kind = measured_peak()
+    sweep_out = {}
+    for b in sweep:
+        wb = dataclasses.replace(w_ev, budgets=tuple(b for _ in w_ev.budgets))
+        ebb = evict_bytes(wb, L)
+        ms, ks = [], []
+        for i in range(3 + max(10, min(args.steps, 20))):
+            cache.restore(snap)
+            for s_ in range(w.batch):
+                cache.set_budget(s_, b)
+            flush.fill_(1); torch.cuda.synchronize()
+            ev[0].record(); cache.evict(binding.ALL_LAYERS); ev[1].record(); torch.cuda.synchronize()
+            if i >= 3:
+                ms.append(ev[0].elapsed_time(ev[1])); ks.append(cache.evict_timing())
+        bms = ranks.max(mean(ms))
+        bk = {k: ranks.max(mean([x[k] for x in ks])) for k in ks[0]}
+        bdom = "score" if bk["score"] >= bk["compact"] else "compact"
+        gbs = ebb["total"] / (bms * 1e-3) / 1e9
+        sweep_out[str(b)] = {"evict_ms": bms, "gbs": ranks.world * gbs, "frac_of_measured_peak": gbs / peak,
+                             "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS, "kernel_ms": bk,
+                             "dominant_kernel": f"k_{bdom}",
+                             "dominant_gbs": ebb[bdom] / (bk[bdom] * 1e-3) / 1e9, "repetitions": len(ms)}
+    for s_, b in enumerate(w.budgets):
+        cache.set_budget(s_, b)
+    cache.restore(snap)
     status, _ = cache.device_status()
     assert status == 0, f"device status {status}"
 
-    mean = lambda xs: sum(xs) / len(xs)
     evict_ms = ranks.max(mean([r["evict"] for r in res]))
     decode_ms = ranks.max(mean([r["decode"] for r in res]))
     kern = {k: ranks.max(mean([r["kernels"][k] for r in res])) for k in res[0]["kernels"]}
@@ -348,18 +402,16 @@ def run_ours(args):
     tok_s = N * w.batch * T / (decode_ms * 1e-3) if T else 0.0
     e_evict = ranks.max(mean([r["h2d"] + r["evict"] for r in e2e_res]))
     e_decode = ranks.max(mean([r["decode"] for r in e2e_res]))
-    peak, peak_kind = measured_peak()
     dom = "score" if kern["score"] >= kern["compact"] else "compact"
     dom_bytes = eb[dom]
     achieved = dom_bytes / (kern[dom] * 1e-3) / 1e9
-    # DRAM traffic of the dominant kernel from its ncu capture on a 4-layer slice of this workload
-    # (profiles/k_score_cfg3_4layers.md, profiles/k_compact_cfg3_4layers.md), scaled by the units of the launch:
-    # 616.2 B per scored pair; 1174 B (read + write) per kept pair at B = 8192 only.
+    # DRAM traffic of the dominant kernel: measured per unit by its ncu capture on a slice of this workload and
+    # scaled to the launch by the units it processes (scored pairs, kept pairs).
     traffic = args.traffic
     if traffic is None and args.config == 3:
         pairs = L * w.num_kv_heads * sum(n for n, b in zip(w.lens, w.budgets) if n > b)
         kept = L * w.num_kv_heads * sum(b for n, b in zip(w.lens, w.budgets) if n > b)
-        traffic = 616.2 * pairs if dom == "score" else (1174.0 * kept if max(w.budgets) == 8192 else None)
+        traffic = profiled_traffic(f"k_{dom}", pairs if dom == "score" else kept, max(w.budgets))
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": N, "steps": args.steps, "warmup": args.warmup,
@@ -380,12 +432,14 @@ def run_ours(args):
         "decode_attn_gbs": N * dec_bytes / (decode_ms * 1e-3) / 1e9 if T else 0.0,
         "decode_attn_frac_of_measured_peak": dec_bytes / (decode_ms * 1e-3) / 1e9 / peak if T else 0.0,
         "decode_us_per_layer_launch": 1e3 * decode_ms / (T * L) if T else 0.0,
+        "decode_note": "attention side only: one launch of append + GQA attention per layer and token "
+                       "(fkv_append_decode_attn), each ordered after the one before; no projections, MLP or sampling",
+        "decode_overlapped_us_per_layer_launch": 1e3 * over_ms,
+        "decode_overlapped_tokens_per_s": N * w.batch / (over_ms * L * 1e-3) if over_ms else 0.0,
+        "decode_overlapped_note": "fkv_decode_step: all layers' k / v / q given up front, consecutive layers' "
+                                  "launches overlap",
         "decode_graph_us_per_layer_launch": 1e3 * graph_ms,
         "decode_graph_tokens_per_s": N * w.batch / (graph_ms * L * 1e-3) if graph_ms else 0.0,
-        "decode_serialised_us_per_layer_launch": 1e3 * serial_ms,
-        "decode_serialised_tokens_per_s": N * w.batch / (serial_ms * L * 1e-3) if serial_ms else 0.0,
-        "decode_note": "attention side only (append + GQA attention, one launch per layer, layers of a token "
-                       "overlap); no projections, MLP or sampling",
         "roofline": {"bound": "hbm", "kernel": f"k_{dom}", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic},
         "e2e": {"value": N * eb["total"] / (e_evict * 1e-3) / 1e9, "unit": UNIT,
@@ -395,6 +449,12 @@ def run_ours(args):
                 "note": "pinned-host decode inputs copied in before the eviction, attention outputs copied out"},
         "gpu_launches": launches, "clocks": clocks,
     }
+    if sweep_out:
+        main = {"evict_ms": evict_ms, "gbs": value, "frac_of_measured_peak": value / N / peak,
+                "frac_of_nominal_8TBps": value / N / NOMINAL_HBM_GBS, "kernel_ms": kern, "dominant_kernel": f"k_{dom}",
+                "dominant_gbs": achieved, "repetitions": args.steps}
+        sweep_out[str(max(w.budgets))] = main
+        line["budget_sweep"] = {k: sweep_out[k] for k in sorted(sweep_out, key=int)}
     if ranks.rank == 0 and N == 1 and not args.no_cpu_baseline:
         smp = oracle_sample(w_ev)
         line["cpu_baseline"] = {
@@ -419,6 +479,7 @@ def main():
     ap.add_argument("--feature-window", type=int, default=0,
                     help="record the decode queries and maintain the attention features (config 2: e.g. 128)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the budget sweep of the default run")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per launch of the dominant kernel")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -53,7 +53,7 @@ struct SmemOptIn {
 };
 
 struct Layout {
-  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, att_part, att_tickets, hist_q, hist_mp, hist_n, hist_cnt, total;
+  size_t pool, free_stack, ctrl, planhdr, pt, pt_new, len, budget, sp, scores, idx, plan, work, tile1, seq_tickets, seq_fail, att_part, att_tickets, hist_q, hist_mp, hist_n, hist_cnt, total;
   int cap, max_pages, num_pages, page_bytes, F, att_smax, sp_stride, sp_off_wf, sp_off_b1, sp_off_w2, sp_off_b2;
 };
 
@@ -105,6 +105,7 @@ Layout make_layout(const fkv_config &c) {
   L.work = take(nseg * 4);
   L.tile1 = take((nseg + 1) * 4);
   L.seq_tickets = take((size_t)c.num_layers * c.max_batch * 4);
+  L.seq_fail = take((size_t)c.num_layers * c.max_batch * 4);
   // Split-K attention: up to att_smax splits per segment (enough for a few CTAs per SM at this batch size).
   L.att_smax = std::max(1, std::min(kMaxSplits, 512 / (c.max_batch * c.num_kv_heads)));
   L.att_part = take(nseg * L.att_smax * c.group_size * (D + 4) * 4);
@@ -278,7 +279,7 @@ int launch_attend_t(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cud
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = pdl ? 1 : 0;
+  cfg.numAttrs = (pdl || a->wait_first) ? 1 : 0;
   FKV_CUDA(cudaLaunchKernelEx(&cfg, kern, c->ctx, *a));
   ++c->launches;
   return FKV_OK;
@@ -299,10 +300,12 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
     const int n = c->h_len[(size_t)layer * batch + s] + ((app && (!seq_mask || ((seq_mask >> s) & 1ull))) ? 1 : 0);
     maxpages = std::max(maxpages, (n + kPage - 1) / kPage);
   }
-  // Splits per segment: CTAs for about three quarters of the SMs per launch (consecutive launches of a decode
-  // step share the SMs, three CTAs fit on one), at least kAttendMinPages pages each.
+  // Splits per segment, at least kAttendMinPages pages each.  A launch of a decode step shares the SMs with the
+  // launches next to it (three CTAs fit on one): CTAs for about three quarters of the SMs.  A launch on its own
+  // has the GPU to itself: CTAs for every slot, so that the most bytes are in flight from the start.
   const int nseg = batch * Hkv;
-  int splits = std::min(c->lay.att_smax, std::max(1, (c->sm_count * 3 / 4 + nseg / 2) / nseg));
+  const int want_ctas = pdl ? c->sm_count * 3 / 4 : c->sm_count * 3;
+  int splits = std::min(c->lay.att_smax, std::max(1, (want_ctas + nseg / 2) / nseg));
   splits = std::max(1, std::min(splits, maxpages / kAttendMinPages));
   const int pps = std::max(1, (maxpages + splits - 1) / splits);
   if (scale == 0.f) scale = 1.f / sqrtf((float)D);
@@ -311,6 +314,7 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
   a.layer = layer; a.q = (const __nv_bfloat16 *)q; a.out = (__nv_bfloat16 *)out;
   a.scale_log2 = scale * 1.4426950408889634f; a.pps = pps; a.append = app ? 1 : 0;
   a.k_new = (const uint8_t *)k_new; a.v_new = (const uint8_t *)v_new; a.pos_new = pos; a.seq_mask = seq_mask;
+  a.wait_first = pdl ? 0 : 1;
   const int rc = attend_dispatch(c, &a, splits, pdl, st);
   if (rc) return rc;
   if (app)
@@ -352,6 +356,7 @@ int fkv_init_cache(const fkv_config *cfg, void *dev_workspace, size_t bytes, voi
   x.scores = (float *)(ws + L.scores); x.idx = (int *)(ws + L.idx); x.plan = (SegPlan *)(ws + L.plan);
   x.work = (int *)(ws + L.work); x.tile1_start = (int *)(ws + L.tile1);
   x.seq_tickets = (int *)(ws + L.seq_tickets);
+  x.seq_fail = (int *)(ws + L.seq_fail);
   x.att_part = (float *)(ws + L.att_part); x.att_tickets = (int *)(ws + L.att_tickets); x.att_smax = L.att_smax;
   x.hist_w = cfg->feature_window; x.hist_q = ws + L.hist_q; x.hist_mp = (float *)(ws + L.hist_mp); x.hist_wp = (cfg->feature_window + 15) & ~15;
   x.hist_n = (int *)(ws + L.hist_n); x.hist_cnt = (int *)(ws + L.hist_cnt);

@@ -72,6 +72,8 @@ struct AttendArgs {
   const uint8_t *k_new, *v_new;  // [batch][Hkv][D] bf16
   const int32_t *pos_new;   // [batch] or null (last position + 1)
   unsigned long long seq_mask;   // sequences that append (0 = all)
+  int wait_first;           // 1: the grid was launched with the programmatic attribute but depends on everything
+                            // before it: wait for the launch before it ahead of the first global read
 };
 
 // The CTA-wide barrier, for the place where the producer warp and the consumer warps meet from different branches.
@@ -188,6 +190,10 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   const int y = blockIdx.y, seq = y / c.Hkv, head = y % c.Hkv, G = c.G;
   const int S = gridDim.x, rank = blockIdx.x;   // splits of the segment, and this CTA's
   const int seg = seg_of(c, a.layer, seq, head);
+  // A launch that depends on all earlier work (the per-layer entry points: the caller's q, k, v come from the
+  // kernel before) still carries the programmatic attribute, so that the grid is scheduled and set up while
+  // that kernel drains; it then waits here, before it reads anything, and is ordered like an ordinary launch.
+  if (a.wait_first) griddep_wait();
   // The producer warp asks for its first page-table entries before the length is known, at the place the host's
   // pages-per-split figure puts them (entries past the segment's pages are never used), so that the two reads
   // overlap instead of following one another.
@@ -269,11 +275,16 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
       // The new pair goes to slot n_old of the page record (and, below, into the consumer's copy of the page).
       int npid = -1;
       if (fresh) {
+        // A fresh page for this head.  If there is none, the append of the whole sequence is abandoned: the
+        // launch's last CTA then leaves the length of every head alone.  Pages that sibling heads did take sit
+        // in their page tables past the length, unused; with the pool empty no eviction can run either, so
+        // the way on is fkv_reset, which rebuilds the free stack.
         if (lane == 0) {
           const int old = atomicSub(&c.ctrl[CTRL_FREE_TOP], 1);
           if (old < 1) {
             atomicAdd(&c.ctrl[CTRL_FREE_TOP], 1);
             set_status(c, kDevPoolExhausted);
+            atomicOr(&c.seq_fail[a.layer * c.batch + seq], 1);
           } else {
             npid = __ldcg(c.free_stack + old - 1);
             ptrow[npages - 1] = npid;
@@ -524,15 +535,21 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
 
   // ---- the length grows once every CTA of the sequence (all heads, all splits) has read the old one ----
   if (app && tid == 0) {
-    const int total = (int)gridDim.x * c.Hkv;
-    int *ticket = &c.seq_tickets[a.layer * c.batch + seq];
+    const int total = (int)gridDim.x * c.Hkv, ls = a.layer * c.batch + seq;
+    int *ticket = &c.seq_tickets[ls];
+    __threadfence();   // this CTA's page-table and failure writes come before its ticket
     const int tk = atomicAdd(ticket, 1);
     if (tk == total - 1) {
       *ticket = 0;
-      c.len[a.layer * c.batch + seq] = n_old + 1;
-      if (rec) {
-        c.hist_n[(size_t)(a.layer * c.batch + seq) * c.hist_w + hcnt % c.hist_w] = n_old + 1;
-        c.hist_cnt[a.layer * c.batch + seq] = hcnt + 1;
+      __threadfence();
+      if ((n_old % kPage) == 0 && atomicExch(&c.seq_fail[ls], 0) != 0) {
+        // a head found no free page: no head's length moves, the token is not recorded
+      } else {
+        c.len[ls] = n_old + 1;
+        if (rec) {
+          c.hist_n[(size_t)ls * c.hist_w + hcnt % c.hist_w] = n_old + 1;
+          c.hist_cnt[ls] = hcnt + 1;
+        }
       }
     }
   }

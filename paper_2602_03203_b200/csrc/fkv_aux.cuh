@@ -14,6 +14,7 @@ __global__ void k_reset(Ctx c) {
   for (int i = t0; i < c.L * c.batch; i += stride) c.len[i] = 0;
   for (int i = t0; i < c.L * c.batch; i += stride) c.seq_tickets[i] = 0;
   for (int i = t0; i < c.L * c.batch * c.Hkv; i += stride) c.att_tickets[i] = 0;
+  for (int i = t0; i < c.L * c.batch; i += stride) c.seq_fail[i] = 0;
   if (c.hist_w)
     for (int i = t0; i < c.L * c.batch; i += stride) c.hist_cnt[i] = 0;
   if (t0 == 0) {

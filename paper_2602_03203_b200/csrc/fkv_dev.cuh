@@ -62,6 +62,7 @@ struct Ctx {
   int *tile1_start;  // prefix of score tiles over the work list
   int *planhdr;
   int *seq_tickets;  // [L][batch]
+  int *seq_fail;     // [L][batch]: set by a head whose append found no free page; read and cleared by the launch's last CTA
   // Split-K attention: partial results [L*batch*Hkv][att_smax][G][D + 4] fp32 and one arrival counter per segment.
   float *att_part;
   int *att_tickets;

@@ -508,6 +508,44 @@ def test_errors_are_status_codes():
     assert big.device_status()[0] == 0
 
 
+@pytest.mark.parametrize("free_pages", [0, 1])
+def test_fused_append_without_free_pages_moves_no_head(free_pages):
+    # A sequence whose length is a multiple of the page size needs a fresh page on EVERY head for its next
+    # pair.  With none free (or fewer than heads) the append is abandoned for all heads: lengths stay, the
+    # stored rows stay, the pool-exhausted bit is set, and a second attempt changes nothing either.  After
+    # fkv_reset the same cache works again.
+    n0, Hkv, g, D = 32, 2, 4, 64
+    w = wl.Workload("tiny_pool", 1, Hkv, g, D, (n0,), (64,), 0, 21, "normal")
+    c = binding.Cache(1, Hkv, g, D, 1, 64, 128, num_pages=Hkv * (n0 // 16) + free_pages)
+    K, V, A, pos = (t.cuda() for t in wl.layer_inputs(w, 0, 0))
+    c.prefill(0, 0, K, V, A, pos)
+    assert c.device_status() == (0, free_pages)
+    k, v = (t.cuda() for t in wl.new_kv(w, 0, 0))
+    q = wl.queries(w, 0, 0).cuda()
+    for attempt in range(2):
+        c.append_decode_attn(0, k, v, q)
+        status, free = c.device_status()
+        assert status & binding.DEV_POOL_EXHAUSTED and free == 0
+        c.sync_lengths()                                              # the documented step after a device error
+        assert c.lengths(0) == [n0]
+        for h in range(Hkv):                                          # the stored rows are untouched
+            k2, v2, _, p2 = c.export_head(0, 0, h)
+            assert np.array_equal(bits(k2), bits(K[h])) and np.array_equal(bits(v2), bits(V[h]))
+            assert p2.tolist() == list(range(n0))
+    c.reset()
+    assert c.device_status() == (0, Hkv * (n0 // 16) + free_pages)
+    c.prefill(0, 0, K[:, :20].contiguous(), V[:, :20].contiguous(), A[:, :20].contiguous(), pos[:20].contiguous())
+    out = c.append_decode_attn(0, k, v, q)
+    assert c.device_status()[0] == 0 and c.lengths(0) == [21]
+    for h in range(Hkv):
+        k2, v2, _, _ = c.export_head(0, 0, h)
+        assert np.array_equal(bits(k2)[:20], bits(K[h, :20])) and np.array_equal(bits(k2)[20], bits(k)[0, h])
+        ref, ref64 = oracle.attend(bits(q)[0, h * g:(h + 1) * g], bits(k2), bits(v2))
+        err = np.abs(bits_to_f64(bits(out)[0, h * g:(h + 1) * g]) - bits_to_f64(ref))
+        assert np.all(err <= np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64)))
+    c.close()
+
+
 # ------------------------------------------------------------------ the sampled action (Section 3.1, Eq. 2; App. B.2)
 @pytest.mark.parametrize("n,B,R", [(512, 256, 0), (600, 344, 32), (5000, 4744, 0), (4097, 4096, 0), (9000, 8744, 256),
                                    (300, 300, 0), (777, 100, 100), (1000, 600, 0), (40000, 39000, 0), (70001, 60000, 5)])
