@@ -193,11 +193,13 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   // A launch that depends on all earlier work (the per-layer entry points: the caller's q, k, v come from the
   // kernel before) still carries the programmatic attribute, so that the grid is scheduled and set up while
   // that kernel drains; it then waits here, before it reads anything, and is ordered like an ordinary launch.
+  // (Asking the pages into L2 ahead of the wait was measured and set aside: the early traffic slows the kernel
+  // that is still running by more than it saves this one.)
   if (a.wait_first) griddep_wait();
+  int *ptrow = c.pt + (size_t)seg * c.max_pages;
   // The producer warp asks for its first page-table entries before the length is known, at the place the host's
   // pages-per-split figure puts them (entries past the segment's pages are never used), so that the two reads
   // overlap instead of following one another.
-  int *ptrow = c.pt + (size_t)seg * c.max_pages;
   int ptv = 0, ptn = 0;
   if (warp == NCW) {
     const int e = rank * a.pps + lane;
