@@ -106,6 +106,26 @@ def score_feature(A, g, column):
     return phi
 
 
+def score_rkv(K, A, g, lambda_a=0.1, lambda_s=0.9, column=SNAPKV_COLUMN, rows=None):
+    """R-KV baseline score (Appendix E.2; the similarity term is the oracle's own reading, see fkv_oracle.c):
+    lambda_a * (window-8 attention, mean over heads) - lambda_s * max_{j != i} cos(k_i, k_j).
+    K: [n][D] bf16 bits; A: [n][6g].  rows: optional int32 list of pairs to compute (else all)."""
+    K, pK = _c(K, np.uint16)
+    A, pA = _c(A, np.float32)
+    n, D = K.shape
+    assert A.shape == (n, 6 * g)
+    if rows is None:
+        phi = np.empty(n, np.float32)
+        prow, nrows = ctypes.c_void_p(0), 0
+    else:
+        rows, prow = _c(rows, np.int32)
+        nrows = rows.shape[0]
+        phi = np.empty(nrows, np.float32)
+    lib().fkv_oracle_score_rkv(pK, pA, n, D, int(g), int(column), ctypes.c_double(float(lambda_a)),
+                               ctypes.c_double(float(lambda_s)), prow, nrows, phi.ctypes.data_as(ctypes.c_void_p))
+    return phi
+
+
 def golden(A, B, L):
     """Golden Eviction labels of one attention group.  A: [g][T][T] fp32 attention probabilities.
 

@@ -19,6 +19,10 @@
  *   attend   Appendix A, problem set-up: softmax renormalised over the
  *            retained set S, o = sum_{i in S} a_i v_i
  *
+ * Baselines of Appendix E.2 (score_feature: H2O, SnapKV; score_rkv: R-KV - the reading of its
+ * similarity term is this file's own, see the function, and is "parity unpinned" against the authors'
+ * code), the sampled action, the attention features and the Golden-Eviction labels follow below.
+ *
  * Parity status: the scorer ARCHITECTURE is pinned (shapes, order k|v|a, the
  * two affine maps); agreement with the authors' trained checkpoints is
  * "parity unpinned" - the paper prints no worked numeric example and no
@@ -234,6 +238,59 @@ void fkv_oracle_score_feature(const float *A, int n, int g, int column, float *p
     for (int j = 0; j < g; ++j) acc = acc + A[(size_t)i * 6 * g + (size_t)j * 6 + column];
     phi[i] = acc / (float)g;
   }
+}
+
+/*
+ * R-KV baseline of Appendix E.2: "Based on the aforementioned SnapKV, R-KV also takes into account the
+ * redundancy among tokens" - the window attention score and a token-to-token similarity are weighed,
+ * 0.1 and 0.9.  The paper gives the two weights and nothing else; the reading taken here (PARITY
+ * UNPINNED against the authors' code, pinned only as a computation):
+ *   attention term  a_i = the SnapKV score already defined above (window-8 column, mean over the g heads)
+ *   similarity term s_i = max over the OTHER pairs j != i of the cosine between the stored keys,
+ *                         cos(k_i, k_j) = <k_i, k_j> / (|k_i| |k_j|), taken as 0 when either key is the
+ *                         zero vector; s_i = 0 when the segment has a single pair.  A pair is redundant
+ *                         when SOME other pair carries nearly the same key; a mean over thousands of
+ *                         unrelated pairs would wash that out, hence the maximum.
+ *   importance      phi_i = lambda_a * a_i - lambda_s * s_i   (redundancy LOWERS importance; the lowest
+ *                         scores are evicted).  No normalisation of either term.
+ * Doubles throughout, cast to fp32 at the end; the attention term is the fp32 value of
+ * fkv_oracle_score_feature.  rows == NULL: all n pairs, phi[n]; else the nrows listed pairs only,
+ * phi[nrows] (each one is an O(n D) loop, so that long segments can be checked on samples).
+ * K: [n][D] bf16; A: [n][6g].
+ */
+void fkv_oracle_score_rkv(const uint16_t *K, const float *A, int n, int D, int g, int column, double lambda_a,
+                          double lambda_s, const int32_t *rows, int nrows, float *phi) {
+  double *norm = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+  for (int i = 0; i < n; ++i) {
+    double ss = 0.0;
+    for (int c = 0; c < D; ++c) {
+      double x = bf16_to_double(K[(size_t)i * D + c]);
+      ss += x * x;
+    }
+    norm[i] = sqrt(ss);
+  }
+  int count = rows ? nrows : n;
+  for (int r = 0; r < count; ++r) {
+    int i = rows ? rows[r] : r;
+    double s = 0.0;
+    int any = 0;
+    for (int j = 0; j < n; ++j) {
+      if (j == i) continue;
+      double cosv = 0.0;
+      if (norm[i] > 0.0 && norm[j] > 0.0) {
+        double dot = 0.0;
+        for (int c = 0; c < D; ++c) dot += bf16_to_double(K[(size_t)i * D + c]) * bf16_to_double(K[(size_t)j * D + c]);
+        cosv = dot / (norm[i] * norm[j]);
+      }
+      if (!any || cosv > s) s = cosv;
+      any = 1;
+    }
+    float acc = 0.0f;
+    for (int h = 0; h < g; ++h) acc = acc + A[(size_t)i * 6 * g + (size_t)h * 6 + column];
+    float a = acc / (float)g;
+    phi[r] = (float)(lambda_a * (double)a - lambda_s * s);
+  }
+  free(norm);
 }
 
 /*

@@ -465,6 +465,63 @@ def test_feature_column_scores():
     assert oracle.select(oracle.score_feature(A2, 1, oracle.H2O_COLUMN), 3, 0).tolist() == [0, 2, 4]
 
 
+# ---------------------------------------------------------------- R-KV baseline (Appendix E.2; weights 0.1 / 0.9)
+def test_rkv_paper_weights_are_the_defaults():
+    f = _facts()
+    import inspect
+    sig = inspect.signature(oracle.score_rkv)
+    assert sig.parameters["lambda_a"].default == f["rkv_weight_attention"]
+    assert sig.parameters["lambda_s"].default == f["rkv_weight_similarity"]
+
+
+def test_rkv_against_library_cosine_matrix():
+    # Random bf16 keys of a non-square shape: the full cosine matrix from a library matmul in fp64, its
+    # diagonal struck out, row maxima (a transposed operand, a missing norm or a kept diagonal fails).
+    rng = np.random.default_rng(31)
+    n, D, g = 57, 64, 3
+    Kb = f32_to_bits(rng.standard_normal((n, D)) * rng.lognormal(0, 1, (1, D)))
+    A = rng.random((n, 6 * g)).astype(np.float32)
+    K = bits_to_f64(Kb)
+    Kn = K / np.linalg.norm(K, axis=1, keepdims=True)
+    C = Kn @ Kn.T
+    np.fill_diagonal(C, -np.inf)
+    snap = A.reshape(n, g, 6)[:, :, 0].astype(np.float64).mean(1)
+    for la, ls in [(0.1, 0.9), (1.0, 0.0), (0.0, 1.0), (0.3, 2.0)]:
+        phi = oracle.score_rkv(Kb, A, g, la, ls)
+        assert np.allclose(phi, la * snap - ls * C.max(1), rtol=0, atol=2e-7)
+    rows = np.array([5, 0, 56, 5], np.int32)                       # the sampled form gives the same values
+    assert np.array_equal(oracle.score_rkv(Kb, A, g, rows=rows), oracle.score_rkv(Kb, A, g)[rows])
+
+
+def test_rkv_closed_forms():
+    g, D = 2, 64
+    # identical keys: every pair has a twin, similarity 1 for all
+    Kb = np.tile(f32_to_bits(np.linspace(-1, 2, D)[None]), (9, 1))
+    Z = np.zeros((9, 6 * g), np.float32)
+    assert np.allclose(oracle.score_rkv(Kb, Z, g, 0.0, 1.0), -1.0, atol=1e-7)
+    # mutually orthogonal keys (scaled unit vectors): similarity 0 for all, whatever the norms
+    E = np.zeros((5, D)); E[np.arange(5), [3, 9, 17, 40, 63]] = [1.0, -2.0, 0.5, 4.0, 8.0]
+    assert np.array_equal(oracle.score_rkv(f32_to_bits(E), Z[:5], g, 0.0, 1.0), np.zeros(5, np.float32))
+    # opposite keys: cosine -1; with a third, unrelated key the maximum picks the larger one (0)
+    O = np.zeros((2, D)); O[0, 0] = 1.0; O[1, 0] = -3.0
+    assert np.allclose(oracle.score_rkv(f32_to_bits(O), Z[:2], g, 0.0, 1.0), 1.0)      # phi = -(-1)
+    O3 = np.vstack([O, np.eye(1, D, 7)])
+    assert np.allclose(oracle.score_rkv(f32_to_bits(O3), Z[:3], g, 0.0, 1.0), 0.0)
+    # a single pair has no other pair; a zero key has cosine 0 with everything
+    assert oracle.score_rkv(f32_to_bits(np.ones((1, D))), Z[:1], g, 0.0, 1.0).tolist() == [0.0]
+    Zk = np.zeros((3, D)); Zk[1] = 1.0; Zk[2] = 1.0
+    assert np.allclose(oracle.score_rkv(f32_to_bits(Zk), Z[:3], g, 0.0, 1.0), [0.0, -1.0, -1.0])
+    # weight of the similarity term -> 0: the SnapKV score, bit for bit, and so the same kept set
+    rng = np.random.default_rng(32)
+    A = rng.random((40, 6 * g)).astype(np.float32)
+    Kr = f32_to_bits(rng.standard_normal((40, D)))
+    assert np.array_equal(oracle.score_rkv(Kr, A, g, 1.0, 0.0), oracle.score_feature(A, g, oracle.SNAPKV_COLUMN))
+    # the sign: of two pairs with equal attention the one with a near-duplicate elsewhere scores lower
+    Kd = rng.standard_normal((6, D)); Kd[4] = Kd[1] * 1.001
+    phi = oracle.score_rkv(f32_to_bits(Kd), np.ones((6, 6 * g), np.float32), g)
+    assert phi[1] < phi[0] and phi[4] < phi[0] and set(oracle.select(phi, 4, 0).tolist()) == {0, 2, 3, 5}
+
+
 # ---------------------------------------------------------------- Golden Eviction labels (Section 3.2, Eq. 3-5)
 def _golden_brute(A, B, L):
     """Independent statement with numpy slicing and Python sets (not the oracle's loops)."""
