@@ -191,7 +191,7 @@ int fkv_evict_sampled(fkv_cache *c, int layer, const float *noise, int32_t noise
  * (summed in head order, divided by g, fp32): column FKV_FEATURE_CUM_SUM is H2O (cumulative
  * attention), FKV_FEATURE_WINDOW8 is SnapKV as the paper uses it (attention of the final 8 tokens).
  * Selection, compaction and (with a feature window) the feature refresh are those of fkv_evict; no
- * scorer needs to be loaded.  R-KV's redundancy term is not provided.
+ * scorer needs to be loaded.
  */
 #define FKV_FEATURE_WINDOW8 0
 #define FKV_FEATURE_WINDOW16 1
@@ -200,6 +200,24 @@ int fkv_evict_sampled(fkv_cache *c, int layer, const float *noise, int32_t noise
 #define FKV_FEATURE_CUM_SUM 4
 #define FKV_FEATURE_CUM_DECAY 5
 int fkv_evict_by_feature(fkv_cache *c, int layer, int32_t column, void *stream);
+
+/*
+ * evict(layer) with the R-KV baseline score - Appendix E.2: "R-KV also takes into account the redundancy among
+ * tokens": the window attention score and a token-to-token similarity are weighed 0.1 and 0.9.  The paper gives
+ * the weights and no formula; this library's reading:
+ *     score_i = lambda_attn * a_i - lambda_sim * s_i
+ *     a_i = the SnapKV score above (feature FKV_FEATURE_WINDOW8 averaged over the g query heads),
+ *     s_i = the largest cosine between the stored key k_i and the key of ANOTHER pair of the same segment
+ *           (0 if either key is the zero vector, or the segment has one pair),
+ * so a pair with a near-duplicate elsewhere in the cache is evicted before an equally attended unique one.
+ * No normalisation of either term.  Cost: the n x n products of a segment's keys, 2 n^2 D flops, on the tensor
+ * cores.  Features must be finite.  Everything else is as in fkv_evict_by_feature.  FKV_RKV_LAMBDA_* are the
+ * paper's weights.  fkv_score_rkv is the score alone (layout as fkv_score).
+ */
+#define FKV_RKV_LAMBDA_ATTN 0.1f
+#define FKV_RKV_LAMBDA_SIM 0.9f
+int fkv_evict_rkv(fkv_cache *c, int layer, float lambda_attn, float lambda_sim, void *stream);
+int fkv_score_rkv(fkv_cache *c, int layer, float lambda_attn, float lambda_sim, float *scores_out, void *stream);
 
 /*
  * decode_attn(q) - Appendix A: out[s][h] = sum_i softmax_i(scale <q[s][h], k_i>) v_i

@@ -26,7 +26,8 @@ EXPORTS = ["fkv_workspace_bytes", "fkv_init_cache", "fkv_destroy", "fkv_reset", 
            "fkv_prefill", "fkv_append", "fkv_set_features", "fkv_evict", "fkv_decode_attn", "fkv_score", "fkv_select",
            "fkv_compact", "fkv_score_stride", "fkv_export_head", "fkv_get_lengths", "fkv_device_status",
            "fkv_launch_count", "fkv_last_cuda_error", "fkv_sync_lengths", "fkv_set_timing", "fkv_get_evict_timing",
-           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled", "fkv_update_features", "fkv_evict_by_feature", "fkv_golden_steps", "fkv_golden_eviction", "fkv_golden_select"]
+           "fkv_decode_step", "fkv_decode_attn_dense_noalloc", "fkv_append_decode_attn", "fkv_evict_sampled", "fkv_select_sampled", "fkv_update_features", "fkv_evict_by_feature", "fkv_golden_steps", "fkv_golden_eviction", "fkv_golden_select",
+           "fkv_evict_rkv", "fkv_score_rkv"]
 
 
 class FkvConfig(ctypes.Structure):
@@ -178,6 +179,18 @@ class Cache:
     def evict_by_feature(self, column, layer=ALL_LAYERS):
         """Baseline eviction: score = one feature column (4: H2O cumulative attention, 0: SnapKV last-8 window)."""
         _check(lib().fkv_evict_by_feature(self._h, layer, int(column), _stream()), "fkv_evict_by_feature")
+
+    def evict_rkv(self, layer=ALL_LAYERS, lambda_attn=0.1, lambda_sim=0.9):
+        """Baseline eviction by the R-KV score: lambda_attn * window attention - lambda_sim * max cosine to another key."""
+        _check(lib().fkv_evict_rkv(self._h, layer, ctypes.c_float(lambda_attn), ctypes.c_float(lambda_sim), _stream()),
+               "fkv_evict_rkv")
+
+    def score_rkv(self, layer, lambda_attn=0.1, lambda_sim=0.9, out=None):
+        if out is None:
+            out = torch.zeros((self.cfg.max_batch, self.cfg.num_kv_heads, self.cap), dtype=torch.float32, device="cuda")
+        _check(lib().fkv_score_rkv(self._h, layer, ctypes.c_float(lambda_attn), ctypes.c_float(lambda_sim),
+                                   _ptr(out, torch.float32), _stream()), "fkv_score_rkv")
+        return out
 
     def decode_attn(self, layer, q, out=None, scale=0.0):
         if out is None:

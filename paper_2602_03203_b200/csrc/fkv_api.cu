@@ -20,6 +20,7 @@
 #include "fkv_dev.cuh"
 #include "fkv_features.cuh"
 #include "fkv_golden.cuh"
+#include "fkv_rkv.cuh"
 #include "fkv_score.cuh"
 #include "fkv_select.cuh"
 
@@ -251,6 +252,31 @@ int launch_features(fkv_cache *c, int max_old, int nwork_bound, cudaStream_t st)
   const float scale_log2 = c->feature_scale * 1.4426950408889634f;
   return c->cfg.head_dim == 128 ? launch_features_t<128>(c, max_old, nwork_bound, scale_log2, st)
                                 : launch_features_t<64>(c, max_old, nwork_bound, scale_log2, st);
+}
+
+// R-KV baseline scores of the segments on the work list (after a k_plan): the attention term and the reciprocal
+// key norms first (the index scratch holds the norms until the selection overwrites it), then the n x n
+// contraction.  Work items sit on grid.x (no 65535 limit).
+template <int D>
+int launch_rkv_t(fkv_cache *c, float *out, int seg_base, int max_old, int nwork_bound, long long tiles, float la, float ls,
+                 cudaStream_t st) {
+  if (max_old <= 0 || nwork_bound <= 0) return FKV_OK;
+  float *rn = reinterpret_cast<float *>(c->ctx.idx);
+  k_rkv_prepare<D><<<dim3(nwork_bound, (max_old + 127) / 128), 128, 0, st>>>(c->ctx, out, rn, seg_base,
+                                                                             FKV_FEATURE_WINDOW8);
+  FKV_LAUNCHED(c);
+  const size_t smem = RkvSmem::bytes(D);
+  static SmemOptIn opt_in;
+  FKV_CUDA(opt_in.ensure(k_rkv_score<D>, smem));
+  const int grid = (int)std::max<long long>(1, std::min<long long>(c->sm_count, tiles));
+  k_rkv_score<D><<<grid, kRkvThreads, smem, st>>>(c->ctx, out, rn, seg_base, la, ls);
+  FKV_LAUNCHED(c);
+  return FKV_OK;
+}
+int launch_rkv(fkv_cache *c, float *out, int seg_base, int max_old, int nwork_bound, long long tiles, float la, float ls,
+               cudaStream_t st) {
+  return c->cfg.head_dim == 128 ? launch_rkv_t<128>(c, out, seg_base, max_old, nwork_bound, tiles, la, ls, st)
+                                : launch_rkv_t<64>(c, out, seg_base, max_old, nwork_bound, tiles, la, ls, st);
 }
 
 int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, int nwork_bound, cudaStream_t st) {
@@ -539,7 +565,10 @@ static int sampled_candidates(int n, int B, int R) {
   return std::min(2 * (n - B), n - std::min(R, B));
 }
 
-static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_stride, int feature_column, void *stream) {
+// score_kind: -1 the learned scorer, 0..5 a feature column (baseline), kScoreRkv the R-KV baseline with its two weights.
+constexpr int kScoreRkv = 100;
+static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_stride, int feature_column, float rkv_a,
+                      float rkv_s, void *stream) {
   if (!c || (layer != FKV_ALL_LAYERS && !layer_ok(c, layer))) return FKV_ERR_INVALID_ARG;
   const int l0 = layer == FKV_ALL_LAYERS ? 0 : layer, l1 = layer == FKV_ALL_LAYERS ? c->cfg.num_layers : layer + 1;
   const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
@@ -573,6 +602,8 @@ static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_str
   int rc = FKV_OK;
   if (feature_column < 0) {
     rc = launch_score_any(c, c->ctx.scores, 0, (int)std::min<long long>(tiles, 1 << 30), st);
+  } else if (feature_column == kScoreRkv) {
+    rc = launch_rkv(c, c->ctx.scores, 0, max_old, nactive, tiles, rkv_a, rkv_s, st);
   } else {   // a baseline: the score is a feature column
     k_score_feature<<<dim3((max_old + 127) / 128, nactive), 128, 0, st>>>(c->ctx, c->ctx.scores, 0, feature_column);
     FKV_LAUNCHED(c);
@@ -604,16 +635,39 @@ static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_str
   return FKV_OK;
 }
 
-int fkv_evict(fkv_cache *c, int layer, void *stream) { return evict_impl(c, layer, nullptr, 0, -1, stream); }
+int fkv_evict(fkv_cache *c, int layer, void *stream) { return evict_impl(c, layer, nullptr, 0, -1, 0.f, 0.f, stream); }
 
 int fkv_evict_by_feature(fkv_cache *c, int layer, int32_t column, void *stream) {
   if (column < 0 || column > 5) return FKV_ERR_INVALID_ARG;
-  return evict_impl(c, layer, nullptr, 0, column, stream);
+  return evict_impl(c, layer, nullptr, 0, column, 0.f, 0.f, stream);
+}
+
+int fkv_evict_rkv(fkv_cache *c, int layer, float lambda_attn, float lambda_sim, void *stream) {
+  if (!std::isfinite(lambda_attn) || !std::isfinite(lambda_sim)) return FKV_ERR_INVALID_ARG;
+  return evict_impl(c, layer, nullptr, 0, kScoreRkv, lambda_attn, lambda_sim, stream);
+}
+
+int fkv_score_rkv(fkv_cache *c, int layer, float lambda_attn, float lambda_sim, float *scores_out, void *stream) {
+  if (!c || !layer_ok(c, layer) || !scores_out || !std::isfinite(lambda_attn) || !std::isfinite(lambda_sim))
+    return FKV_ERR_INVALID_ARG;
+  const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads;
+  long long tiles = 0;
+  int max_old = 0;
+  for (int s = 0; s < batch; ++s) {
+    const int n = c->h_len[(size_t)layer * batch + s];
+    tiles += (long long)Hkv * ((n + kScorePPS * kPage - 1) / (kScorePPS * kPage));
+    max_old = std::max(max_old, n);
+  }
+  if (tiles == 0) return FKV_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  k_plan<<<1, 1024, 0, st>>>(c->ctx, layer, layer + 1, PLAN_SCORE_ALL, kScorePPS * kPage, nullptr);
+  FKV_LAUNCHED(c);
+  return launch_rkv(c, scores_out, layer * batch * Hkv, max_old, batch * Hkv, tiles, lambda_attn, lambda_sim, st);
 }
 
 int fkv_evict_sampled(fkv_cache *c, int layer, const float *noise, int32_t noise_stride, void *stream) {
   if (!noise || noise_stride < 1) return FKV_ERR_INVALID_ARG;
-  return evict_impl(c, layer, noise, noise_stride, -1, stream);
+  return evict_impl(c, layer, noise, noise_stride, -1, 0.f, 0.f, stream);
 }
 
 int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream) {
