@@ -390,6 +390,32 @@ def run_ours(args):
                              "dominant_gbs": ebb[bdom] / (bk[bdom] * 1e-3) / 1e9, "repetitions": len(ms)}
     for s_, b in enumerate(w.budgets):
         cache.set_budget(s_, b)
+    # The baseline scores of Appendix E.2 on the same select / compact machinery: H2O and SnapKV read one feature
+    # column; R-KV adds the n x n key-similarity contraction (2 n^2 D flops per segment, tensor cores).
+    base_out = {}
+    if not args.no_baselines:
+        n2 = sum(float(n) * n for n, b in zip(w_ev.lens, w_ev.budgets) if n > b)
+        rkv_flops = 2.0 * n2 * w.head_dim * L * w.num_kv_heads
+        for name, fn in (("h2o", lambda: cache.evict_by_feature(4)), ("snapkv", lambda: cache.evict_by_feature(0)),
+                         ("rkv", lambda: cache.evict_rkv())):
+            ms, ks = [], []
+            for i in range(4):
+                cache.restore(snap); flush.fill_(1); torch.cuda.synchronize()
+                if chunk_mode:
+                    for t in range(T):
+                        cache.decode_step(kd[t], vd[t], qd[t], od[t])
+                ev[0].record(); fn(); ev[1].record(); torch.cuda.synchronize()
+                if i >= 1:
+                    ms.append(ev[0].elapsed_time(ev[1])); ks.append(cache.evict_timing()["score"])
+            base_out[name] = {"evict_ms": ranks.max(mean(ms)), "score_ms": ranks.max(mean(ks))}
+        bf16_peak = None
+        try:
+            bf16_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"])
+        except Exception:
+            pass
+        tf = rkv_flops / (base_out["rkv"]["score_ms"] * 1e-3) / 1e12
+        base_out["rkv"].update({"tflops": tf, "frac_of_measured_bf16_sustained": tf / bf16_peak if bf16_peak else None,
+                                "flops": rkv_flops})
     cache.restore(snap)
     status, _ = cache.device_status()
     assert status == 0, f"device status {status}"
@@ -449,6 +475,8 @@ def run_ours(args):
                 "note": "pinned-host decode inputs copied in before the eviction, attention outputs copied out"},
         "gpu_launches": launches, "clocks": clocks,
     }
+    if base_out:
+        line["baseline_scorers"] = base_out
     if sweep_out:
         main = {"evict_ms": evict_ms, "gbs": value, "frac_of_measured_peak": value / N / peak,
                 "frac_of_nominal_8TBps": value / N / NOMINAL_HBM_GBS, "kernel_ms": kern, "dominant_kernel": f"k_{dom}",
@@ -480,6 +508,7 @@ def main():
                     help="record the decode queries and maintain the attention features (config 2: e.g. 128)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the budget sweep of the default run")
+    ap.add_argument("--no-baselines", action="store_true", help="skip the H2O / SnapKV / R-KV eviction timings")
     ap.add_argument("--traffic", type=float, default=None, help="ncu DRAM bytes per launch of the dominant kernel")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

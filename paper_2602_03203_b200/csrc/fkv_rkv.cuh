@@ -154,9 +154,17 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, float *out,
         }
       }
     };
-    FeatRing br{0, 0};
+    // The column tiles are copied two ahead: the copies of tile j are issued before those of tile j - 2 are waited
+    // for (a copy from L2 takes longer than the multiplies of a tile), and a tile is handed over - this thread's
+    // copies complete, made visible to the tensor core's reads, one arrival - two tiles after it was asked for.
+    FeatRing br{0, 0}, done{0, 0};
     int nu = 0, jr = 0;   // units so far (phase of the A barriers); ring slot of the next column tile's norms
     bool ok = true;
+    auto hand_over = [&]() {
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&b_full[done.i]));
+      done.next(NST);
+    };
     for (int t = t0; t < t1 && ok;) {
       const int took = rkv_unit(c, t, t1, w, u);
       if (!mbar_wait_warp(smem_u32(a_empty), (nu & 1) ^ 1)) { set_status(c, kDevWaitTimeout); break; }
@@ -164,17 +172,24 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, float *out,
       cp_async_wait_all();
       fence_proxy_async();
       mbar_arrive(smem_u32(a_full));
+      int inflight = 0;
       for (int j = 0; j < u.ntj; ++j) {
         if (!mbar_wait_warp(smem_u32(&b_empty[br.i]), br.ph ^ 1)) { set_status(c, kDevWaitTimeout); ok = false; break; }
         copy_tile(smem_u32(Bt + br.i * tb), j * 8);
         if (p < 32 && j * 128 + p * 4 < c.cap)   // this tile's reciprocal norms (entries past the segment's end are masked later)
           cp_async16(smem_u32(Rn + jr * 128 + p * 4), rn + (size_t)w.seg * c.cap + j * 128 + p * 4);
-        cp_async_wait_all();
-        fence_proxy_async();
-        mbar_arrive(smem_u32(&b_full[br.i]));
+        cp_async_commit();
         br.next(NST);
         if (++jr == NR) jr = 0;
+        if (++inflight == 3) {
+          cp_async_wait_pending<2>();
+          hand_over();
+          --inflight;
+        }
       }
+      // The last tiles of the unit (on a failed wait too: nothing may be in flight at the exit).
+      cp_async_wait_pending<0>();
+      for (; inflight > 0 && ok; --inflight) hand_over();
       ++nu;
       t += took;
     }
