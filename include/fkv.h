@@ -73,7 +73,7 @@ typedef struct {
   int32_t num_kv_heads;
   int32_t group_size;          /* g, 1..8 */
   int32_t head_dim;            /* D, 64 or 128 */
-  int32_t max_batch;           /* sequences */
+  int32_t max_batch;           /* sequences, at most 256 (the efficiency table of Section 4.3 runs up to 96) */
   int32_t page_size;           /* pairs per page; must be 16 */
   int32_t scorer_hidden;       /* H; must be 16 (Section 4.1) */
   int32_t activation;          /* FKV_ACT_* */
@@ -140,10 +140,11 @@ int fkv_prefill(fkv_cache *c, int layer, int seq, const void *k, const void *v, 
  * append(k, v) - Section 3.1: one new pair per sequence and KV head of `layer`.
  * k, v: dev [max_batch][Hkv][D] bf16; pos: dev [max_batch] int32 token
  * positions, or NULL: the position after the last stored one (0 for an empty
- * segment).  The feature row of the new pair is zero.  seq_mask: host bitmask
- * of the sequences that take part (bit s), 0 = all.
+ * segment).  The feature row of the new pair is zero.  seq_mask: host bit
+ * array of the sequences that take part, (max_batch + 63) / 64 words, bit
+ * s % 64 of word s / 64; NULL = all.  It is read before the call returns.
  */
-int fkv_append(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, uint64_t seq_mask,
+int fkv_append(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, const uint64_t *seq_mask,
                void *stream);
 
 /*
@@ -235,7 +236,7 @@ int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float sca
  * one after the other.
  */
 int fkv_append_decode_attn(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos,
-                           uint64_t seq_mask, const void *q, void *out, float scale, void *stream);
+                           const uint64_t *seq_mask, const void *q, void *out, float scale, void *stream);
 
 /*
  * One decode token through every layer, in layer order: for l = 0 .. L-1,

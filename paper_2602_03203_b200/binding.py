@@ -57,9 +57,9 @@ def lib():
         _lib.fkv_last_cuda_error.restype = ctypes.c_char_p
         vp, i32, u64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint64, ctypes.c_float
         # Declared argument types for the per-token calls: plain ints and floats are converted by ctypes itself.
-        _lib.fkv_append.argtypes = [vp, i32, vp, vp, vp, u64, vp]
+        _lib.fkv_append.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         _lib.fkv_decode_attn.argtypes = [vp, i32, vp, vp, f32, vp]
-        _lib.fkv_append_decode_attn.argtypes = [vp, i32, vp, vp, vp, u64, vp, vp, f32, vp]
+        _lib.fkv_append_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, f32, vp]
         _lib.fkv_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, f32, vp]
         _lib.fkv_evict.argtypes = [vp, i32, vp]
     return _lib
@@ -84,6 +84,16 @@ try:   # the raw handle of torch's current stream without building a Stream obje
     _raw_stream = torch._C._cuda_getCurrentRawStream
 except AttributeError:   # pragma: no cover
     _raw_stream = None
+
+
+def _mask(seq_mask, max_batch):
+    """A Python integer with bit s set for every sequence that takes part (0 or None: all) as the host bit
+    array the library reads: (array or None to keep alive, pointer)."""
+    if not seq_mask:
+        return None, ctypes.c_void_p(0)
+    words = (max_batch + 63) // 64
+    arr = (ctypes.c_uint64 * words)(*[(seq_mask >> (64 * i)) & 0xFFFFFFFFFFFFFFFF for i in range(words)])
+    return arr, ctypes.cast(arr, ctypes.c_void_p)
 
 
 def _stream():
@@ -165,8 +175,9 @@ class Cache:
 
     # -- the four calls of the path
     def append(self, layer, k, v, pos=None, seq_mask=0):
+        keep, m = _mask(seq_mask, self.cfg.max_batch)
         _check(lib().fkv_append(self._h, layer, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
-                                _ptr(pos, torch.int32), seq_mask, _stream()), "fkv_append")
+                                _ptr(pos, torch.int32), m, _stream()), "fkv_append")
 
     def evict(self, layer=ALL_LAYERS):
         _check(lib().fkv_evict(self._h, layer, _stream()), "fkv_evict")
@@ -203,10 +214,28 @@ class Cache:
         """append(k, v) then decode_attn(q) on one layer, as one launch."""
         if out is None:
             out = torch.empty_like(q)
+        keep, m = _mask(seq_mask, self.cfg.max_batch)
         _check(lib().fkv_append_decode_attn(self._h, layer, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
-                                            _ptr(pos, torch.int32), seq_mask, _ptr(q, torch.bfloat16),
+                                            _ptr(pos, torch.int32), m, _ptr(q, torch.bfloat16),
                                             _ptr(out, torch.bfloat16), scale, _stream()), "fkv_append_decode_attn")
         return out
+
+    def bound_append_decode_attn(self, layer, k, v, q, out, pos=None, seq_mask=0, scale=0.0):
+        """The same call with its arguments checked and marshalled once: returns a function of no arguments that
+        enqueues append + attention on `layer` over these (fixed) tensors on the stream current at THIS call, and
+        raises on a non-zero status.  For decode loops that reuse their k / v / q / out buffers, where the
+        per-call conversion of ten arguments costs more host time than the kernel takes."""
+        fn = lib().fkv_append_decode_attn
+        mask_arr, m = _mask(seq_mask, self.cfg.max_batch)
+        args = (self._h, layer, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16), _ptr(pos, torch.int32), m,
+                _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16), scale, _stream())
+        keep = (k, v, q, out, pos, mask_arr)   # the tensors stay alive as long as the function does
+
+        def call(_fn=fn, _args=args, _keep=keep):
+            code = _fn(*_args)
+            if code:
+                raise FkvError(code, "fkv_append_decode_attn")
+        return call
 
     def decode_step(self, k, v, q, out=None, pos=None, scale=0.0):
         """One token through all layers: k, v [L][batch][Hkv][D]; q, out [L][batch][Hq][D]."""

@@ -60,7 +60,7 @@ struct Layout {
 
 bool valid_config(const fkv_config *c) {
   if (!c) return false;
-  if (c->num_layers < 1 || c->num_kv_heads < 1 || c->num_kv_heads > 32 || c->max_batch < 1 || c->max_batch > 64)
+  if (c->num_layers < 1 || c->num_kv_heads < 1 || c->num_kv_heads > 32 || c->max_batch < 1 || c->max_batch > kMaxBatch)
     return false;
   if (c->group_size < 1 || c->group_size > 8) return false;
   if (c->head_dim != 64 && c->head_dim != 128) return false;
@@ -176,6 +176,16 @@ int cuda_fail(cudaError_t e) {
     if (e_ != cudaSuccess) return cuda_fail(e_); \
   } while (0)
 
+// The caller's bit array (host, one word per 64 sequences; NULL = every sequence) as the kernels take it.
+SeqMask make_mask(const fkv_cache *c, const uint64_t *bits) {
+  SeqMask m = {};
+  if (bits) {
+    m.use = 1;
+    for (int i = 0; i < (c->cfg.max_batch + 63) / 64; ++i) m.w[i] = bits[i];
+  }
+  return m;
+}
+
 bool layer_ok(const fkv_cache *c, int layer) { return layer >= 0 && layer < c->cfg.num_layers; }
 
 // Page slots of the scorer's ring: as many as fit the shared memory, a multiple of the number of warps (a slot
@@ -280,10 +290,12 @@ int launch_rkv(fkv_cache *c, float *out, int seg_base, int max_old, int nwork_bo
 }
 
 int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, int nwork_bound, cudaStream_t st) {
-  dim3 grid((max_new + kCompactRows - 1) / kCompactRows, nwork_bound);
-  if (grid.x == 0 || grid.y == 0) return FKV_OK;
-  if (c->cfg.head_dim == 128) k_compact<128><<<grid, 256, 0, st>>>(c->ctx, idx, seg_base);
-  else k_compact<64><<<grid, 256, 0, st>>>(c->ctx, idx, seg_base);
+  const int tiles = (max_new + kCompactRows - 1) / kCompactRows;
+  const long long ctas = (long long)nwork_bound * tiles;   // one flat grid: no 65535 limit on the work list
+  if (ctas == 0) return FKV_OK;
+  if (ctas > 0x7fffffffLL) return FKV_ERR_INVALID_ARG;
+  if (c->cfg.head_dim == 128) k_compact<128><<<(unsigned)ctas, 256, 0, st>>>(c->ctx, idx, seg_base, tiles);
+  else k_compact<64><<<(unsigned)ctas, 256, 0, st>>>(c->ctx, idx, seg_base, tiles);
   FKV_LAUNCHED(c);
   return FKV_OK;
 }
@@ -318,12 +330,12 @@ int attend_dispatch(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cud
 
 // Attention over `layer`, with the new pair of every participating sequence appended first when k_new is given.
 int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale, const void *k_new, const void *v_new,
-                  const int32_t *pos, uint64_t seq_mask, bool pdl, cudaStream_t st) {
+                  const int32_t *pos, const SeqMask &seq_mask, bool pdl, cudaStream_t st) {
   const int batch = c->cfg.max_batch, Hkv = c->cfg.num_kv_heads, D = c->cfg.head_dim;
   const bool app = k_new != nullptr;
   int maxpages = 0;
   for (int s = 0; s < batch; ++s) {
-    const int n = c->h_len[(size_t)layer * batch + s] + ((app && (!seq_mask || ((seq_mask >> s) & 1ull))) ? 1 : 0);
+    const int n = c->h_len[(size_t)layer * batch + s] + ((app && seq_mask.has(s)) ? 1 : 0);
     maxpages = std::max(maxpages, (n + kPage - 1) / kPage);
   }
   // Splits per segment: CTAs for about three quarters of the SMs per launch, at least kAttendMinPages pages each.
@@ -346,7 +358,7 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
   if (rc) return rc;
   if (app)
     for (int s = 0; s < batch; ++s)
-      if (!seq_mask || ((seq_mask >> s) & 1ull)) ++c->h_len[(size_t)layer * batch + s];
+      if (seq_mask.has(s)) ++c->h_len[(size_t)layer * batch + s];
   return FKV_OK;
 }
 
@@ -544,18 +556,18 @@ int fkv_set_features(fkv_cache *c, int layer, int seq, const float *feat, void *
   return FKV_OK;
 }
 
-int fkv_append(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, uint64_t seq_mask,
+int fkv_append(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, const uint64_t *seq_mask,
                void *stream) {
   if (!c || !layer_ok(c, layer) || !k || !v) return FKV_ERR_INVALID_ARG;
   const int batch = c->cfg.max_batch;
+  const SeqMask m = make_mask(c, seq_mask);
   for (int s = 0; s < batch; ++s)
-    if ((!seq_mask || ((seq_mask >> s) & 1ull)) && c->h_len[(size_t)layer * batch + s] >= c->lay.cap)
-      return FKV_ERR_CAPACITY;
+    if (m.has(s) && c->h_len[(size_t)layer * batch + s] >= c->lay.cap) return FKV_ERR_CAPACITY;
   k_append<<<batch, 32 * c->cfg.num_kv_heads, 0, (cudaStream_t)stream>>>(c->ctx, layer, (const uint8_t *)k,
-                                                                        (const uint8_t *)v, pos, seq_mask);
+                                                                        (const uint8_t *)v, pos, m);
   FKV_LAUNCHED(c);
   for (int s = 0; s < batch; ++s)
-    if (!seq_mask || ((seq_mask >> s) & 1ull)) ++c->h_len[(size_t)layer * batch + s];
+    if (m.has(s)) ++c->h_len[(size_t)layer * batch + s];
   return FKV_OK;
 }
 
@@ -605,7 +617,7 @@ static int evict_impl(fkv_cache *c, int layer, const float *noise, int noise_str
   } else if (feature_column == kScoreRkv) {
     rc = launch_rkv(c, c->ctx.scores, 0, max_old, nactive, tiles, rkv_a, rkv_s, st);
   } else {   // a baseline: the score is a feature column
-    k_score_feature<<<dim3((max_old + 127) / 128, nactive), 128, 0, st>>>(c->ctx, c->ctx.scores, 0, feature_column);
+    k_score_feature<<<dim3(nactive, (max_old + 127) / 128), 128, 0, st>>>(c->ctx, c->ctx.scores, 0, feature_column);
     FKV_LAUNCHED(c);
   }
   if (rc) return rc;
@@ -672,17 +684,17 @@ int fkv_evict_sampled(fkv_cache *c, int layer, const float *noise, int32_t noise
 
 int fkv_decode_attn(fkv_cache *c, int layer, const void *q, void *out, float scale, void *stream) {
   if (!c || !layer_ok(c, layer) || !q || !out) return FKV_ERR_INVALID_ARG;
-  return launch_attend(c, layer, q, out, scale, nullptr, nullptr, nullptr, 0, false, (cudaStream_t)stream);
+  return launch_attend(c, layer, q, out, scale, nullptr, nullptr, nullptr, make_mask(c, nullptr), false, (cudaStream_t)stream);
 }
 
-int fkv_append_decode_attn(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos, uint64_t seq_mask,
-                           const void *q, void *out, float scale, void *stream) {
+int fkv_append_decode_attn(fkv_cache *c, int layer, const void *k, const void *v, const int32_t *pos,
+                           const uint64_t *seq_mask, const void *q, void *out, float scale, void *stream) {
   if (!c || !layer_ok(c, layer) || !k || !v || !q || !out) return FKV_ERR_INVALID_ARG;
   const int batch = c->cfg.max_batch;
+  const SeqMask m = make_mask(c, seq_mask);
   for (int s = 0; s < batch; ++s)
-    if ((!seq_mask || ((seq_mask >> s) & 1ull)) && c->h_len[(size_t)layer * batch + s] >= c->lay.cap)
-      return FKV_ERR_CAPACITY;
-  return launch_attend(c, layer, q, out, scale, k, v, pos, seq_mask, false, (cudaStream_t)stream);
+    if (m.has(s) && c->h_len[(size_t)layer * batch + s] >= c->lay.cap) return FKV_ERR_CAPACITY;
+  return launch_attend(c, layer, q, out, scale, k, v, pos, m, false, (cudaStream_t)stream);
 }
 
 int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *pos, const void *q, void *out,
@@ -694,11 +706,12 @@ int fkv_decode_step(fkv_cache *c, const void *k, const void *v, const int32_t *p
       if (c->h_len[(size_t)l * batch + s] >= c->lay.cap) return FKV_ERR_CAPACITY;
   const size_t kv_stride = (size_t)batch * c->cfg.num_kv_heads * c->cfg.head_dim * 2;
   const size_t q_stride = kv_stride * c->cfg.group_size;
+  const SeqMask all = make_mask(c, nullptr);
   for (int l = 0; l < c->cfg.num_layers; ++l) {
     // Layer l's launch may run alongside layer l - 1's: each touches only its own layer's cache state and
     // tensors.  Layer 0's launch is ordered after everything before it on the stream, as usual.
     const int rc = launch_attend(c, l, (const uint8_t *)q + l * q_stride, (uint8_t *)out + l * q_stride, scale,
-                                 (const uint8_t *)k + l * kv_stride, (const uint8_t *)v + l * kv_stride, pos, 0, l > 0,
+                                 (const uint8_t *)k + l * kv_stride, (const uint8_t *)v + l * kv_stride, pos, all, l > 0,
                                  (cudaStream_t)stream);
     if (rc) return rc;
   }

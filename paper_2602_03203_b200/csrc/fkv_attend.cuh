@@ -71,7 +71,7 @@ struct AttendArgs {
   int append;               // 1: append k_new / v_new at slot n first (and record the query when the cache keeps a history)
   const uint8_t *k_new, *v_new;  // [batch][Hkv][D] bf16
   const int32_t *pos_new;   // [batch] or null (last position + 1)
-  unsigned long long seq_mask;   // sequences that append (0 = all)
+  SeqMask seq_mask;         // sequences that append
   int wait_first;           // 1: the grid was launched with the programmatic attribute but depends on everything
                             // before it: wait for the launch before it ahead of the first global read
 };
@@ -208,7 +208,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   }
   const int n_old = __ldcg(c.len + a.layer * c.batch + seq);
   // The host refuses an append past the capacity; a replayed launch (CUDA graph) is checked here instead.
-  const bool want = a.append && (!a.seq_mask || ((a.seq_mask >> seq) & 1ull));
+  const bool want = a.append && a.seq_mask.has(seq);
   const bool app = want && n_old < c.cap;
   if (want && !app && tid == 0 && rank == 0) set_status(c, kDevCapacity);
   const int n = n_old + (app ? 1 : 0);

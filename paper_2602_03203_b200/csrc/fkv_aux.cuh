@@ -86,10 +86,10 @@ __global__ void k_export_rows(Ctx c, int layer, int seq, int head, uint8_t *k, u
 // ---------------------------------------------------------------- append
 // grid = batch, block = 32 * Hkv: one warp per KV head writes the new pair at
 // slot n; a new page per head is popped from the free stack when n % 16 == 0.
-__global__ void k_append(Ctx c, int layer, const uint8_t *k, const uint8_t *v, const int32_t *pos, uint64_t seq_mask) {
+__global__ void k_append(Ctx c, int layer, const uint8_t *k, const uint8_t *v, const int32_t *pos, SeqMask seq_mask) {
   __shared__ int s_top;
   const int seq = blockIdx.x, lane = threadIdx.x & 31, h = threadIdx.x >> 5;
-  if (seq_mask && !((seq_mask >> seq) & 1ull)) return;
+  if (!seq_mask.has(seq)) return;
   const int n = c.len[layer * c.batch + seq];
   if (n >= c.cap) {
     if (threadIdx.x == 0) set_status(c, kDevCapacity);

@@ -3,8 +3,8 @@
 // and position id move together from the old pages into fresh pages, so the
 // gather never overwrites a row it still has to read.
 //
-// Roofline: HBM, 2 x (4D + 4F + 4) bytes per kept pair.  grid (tiles of 64
-// output rows, work list).  The CTA first resolves index and page-table
+// Roofline: HBM, 2 x (4D + 4F + 4) bytes per kept pair.  One CTA per (work item,
+// tile of 64 output rows), the tiles of an item on consecutive CTAs.  The CTA first resolves index and page-table
 // lookups for all its rows in one step, then every warp moves 8 rows: all
 // loads first, then all stores, 16 bytes per lane for K and V and one or two
 // 32-bit words per lane for the meta row (features + position, one run).
@@ -18,17 +18,18 @@ constexpr int kCompactRows = 64;  // output rows per CTA (four pages)
 constexpr int kCompactRPW = 8;    // rows per warp, all loaded before any is stored
 
 template <int D>
-__global__ void __launch_bounds__(256) k_compact(Ctx c, const int32_t *idx, int seg_base) {
+__global__ void __launch_bounds__(256) k_compact(Ctx c, const int32_t *idx, int seg_base, int tiles) {
   constexpr int NCH = D / 8;               // 16-byte chunks per K (or V) row
   static_assert(2 * NCH <= 32, "one chunk per lane");
   __shared__ long long s_src[kCompactRows];  // physical source slot (page * 16 + row) or -1
   __shared__ int s_dst[kCompactRows / kPage];
-  if ((int)blockIdx.y >= c.planhdr[PH_NWORK]) return;
-  const int seg = c.work[blockIdx.y];
+  const int wk = blockIdx.x / tiles;   // consecutive CTAs: consecutive row tiles of one work item
+  if (wk >= c.planhdr[PH_NWORK]) return;
+  const int seg = c.work[wk];
   const SegPlan p = c.plan[seg];
   if (!p.active) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int j0 = blockIdx.x * kCompactRows;
+  const int j0 = (blockIdx.x % tiles) * kCompactRows;
   if (j0 >= p.n_new) return;
   // Phase 1: one index and one page-table lookup per output row, all rows of the CTA at once.
   if (threadIdx.x < kCompactRows) {

@@ -77,6 +77,14 @@ struct Ctx {
   int *hist_cnt;       // [L][batch]: queries recorded since the last eviction
 };
 
+// The sequences that take part in an append: bit s of word s / 64; use == 0 means every sequence.
+constexpr int kMaxBatch = 256;
+struct SeqMask {
+  unsigned long long w[kMaxBatch / 64];
+  int use;
+  __host__ __device__ bool has(int s) const { return !use || ((w[s >> 6] >> (s & 63)) & 1ull); }
+};
+
 __device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head) {
   return (layer * c.batch + seq) * c.Hkv + head;
 }

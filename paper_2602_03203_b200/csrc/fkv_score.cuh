@@ -263,12 +263,12 @@ __global__ void __launch_bounds__(NCW * 32, 1) k_score(Ctx c, float *out, int se
 // Baseline scores that need no learned scorer (Appendix E.2): one attention-feature column averaged
 // over the g query heads of the KV head - H2O's cumulative attention (column 4), SnapKV's window of
 // the final 8 tokens (column 0).  The heads are summed in order and divided by g in fp32.
-// grid (tiles of 128 pairs, work list); thread = pair; reads only the meta rows (4F + 4 bytes per pair).
+// grid (work list, tiles of 128 pairs); thread = pair; reads only the meta rows (4F + 4 bytes per pair).
 __global__ void __launch_bounds__(128) k_score_feature(Ctx c, float *out, int seg_base, int column) {
-  if ((int)blockIdx.y >= c.planhdr[PH_NWORK]) return;
-  const int seg = c.work[blockIdx.y];
+  if ((int)blockIdx.x >= c.planhdr[PH_NWORK]) return;
+  const int seg = c.work[blockIdx.x];
   const int n = c.plan[seg].n_old;
-  const int slot = blockIdx.x * 128 + threadIdx.x;
+  const int slot = blockIdx.y * 128 + threadIdx.x;
   if (slot >= n) return;
   const uint8_t *page = c.pool + (size_t)c.pt[(size_t)seg * c.max_pages + slot / kPage] * c.page_bytes;
   const float *f = meta_row(c, page, slot % kPage) + column;

@@ -424,6 +424,40 @@ def test_fused_append_mask_and_decode_step_match_separate_calls():
     assert a.cache.device_status()[0] == 0 and b.cache.device_status()[0] == 0
 
 
+def test_batch_of_96_sequences():
+    # The efficiency table of Section 4.3 runs up to 96 concurrent sequences: more than one 64-bit word of the
+    # sequence mask.  One eviction and masked appends over 96 short sequences of different lengths.
+    rng = np.random.default_rng(96)
+    lens = tuple(int(x) for x in rng.integers(40, 140, 96))
+    w = wl.Workload("b96", 1, 2, 4, 64, lens, tuple(48 for _ in lens), 8, 25, "normal")
+    ld = Loaded(w)
+    scores = npf(ld.cache.score(0))
+    ld.cache.evict(0)
+    assert ld.cache.lengths(0) == [min(48, n) for n in lens]
+    mask = (1 << 95) | (1 << 64) | (1 << 63) | 1 | (1 << 17)
+    k, v = (t.cuda() for t in wl.new_kv(w, 0, 0))
+    q = wl.queries(w, 0, 0).cuda()
+    out = ld.cache.append_decode_attn(0, k, v, q, seq_mask=mask)
+    ld.cache.append(0, k, v, seq_mask=1 << 70)
+    want = [min(48, n) + (1 if (mask >> s) & 1 or s == 70 else 0) for s, n in enumerate(lens)]
+    assert ld.cache.lengths(0) == want
+    g = w.group_size
+    for s in (0, 1, 17, 63, 64, 70, 95):
+        for h in range(2):
+            K, V, A, pos = ld.head(0, s, h)
+            kept = oracle.select(scores[s, h, :lens[s]], 48, 8)
+            k2, v2, _, p2 = ld.export(0, s, h)
+            nk = len(kept)
+            assert np.array_equal(p2[:nk], pos[kept]) and np.array_equal(k2[:nk], K[kept])
+            assert len(p2) == want[s]
+            if (mask >> s) & 1:
+                assert np.array_equal(k2[nk], bits(k)[s, h])
+                ref, ref64 = oracle.attend(bits(q)[s, h * g:(h + 1) * g], k2, v2)
+                err = np.abs(bits_to_f64(bits(out)[s, h * g:(h + 1) * g]) - bits_to_f64(ref))
+                assert np.all(err <= np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64)))
+    assert ld.cache.device_status()[0] == 0
+
+
 # ------------------------------------------------------------------ the decode protocol of Section 3.1
 def test_decode_schedule_sawtooth():
     # cache at B, then L appended tokens -> B + L -> evict back to B, keeping the last L (R = L).
