@@ -56,12 +56,8 @@ __global__ void __launch_bounds__(256) k_golden_suffix_max(float *alpha, int T, 
 __global__ void __launch_bounds__(1024) k_golden_select(const float *alpha, int T, int B, int L, int M,
                                                          int32_t *kept) {
   extern __shared__ __align__(16) uint8_t gsm[];
-  constexpr int kBins = 2048, kLogBins = 11, kPer = 8;
-  __shared__ unsigned s_hist[kBins];
-  __shared__ int s_scan[33];
-  __shared__ unsigned s_red[64];
-  __shared__ unsigned s_bin, s_krem;
-  __shared__ unsigned long long s_wsum[33];
+  constexpr int kPer = 8;
+  __shared__ SelShared<1024> sh;
   int *cache = reinterpret_cast<int *>(gsm);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int per = (B + 1023) / 1024, j0 = min(B, tid * per), j1 = min(B, j0 + per), nm = j1 - j0;
@@ -77,89 +73,21 @@ __global__ void __launch_bounds__(1024) k_golden_select(const float *alpha, int 
       pos[u] = u < nm ? cache[j0 + u] : 0;
       key[u] = u < nm ? score_key(__ldg(a + pos[u])) : 0u;
     }
-    // ---- key window ----
-    uint32_t kmin = 0xffffffffu, kmax = 0u;
-#pragma unroll
-    for (int u = 0; u < kPer; ++u)
-      if (u < nm) { kmin = min(kmin, key[u]); kmax = max(kmax, key[u]); }
-    kmin = __reduce_min_sync(0xffffffffu, kmin);
-    kmax = __reduce_max_sync(0xffffffffu, kmax);
-    if (lane == 0) { s_red[warp] = kmin; s_red[32 + warp] = kmax; }
-    __syncthreads();
-    kmin = __reduce_min_sync(0xffffffffu, s_red[lane]);
-    kmax = __reduce_max_sync(0xffffffffu, s_red[32 + lane]);
-    uint32_t Tk = kmin;
-    unsigned need = (unsigned)k;
-    if (kmin != kmax) {
-      uint32_t lo = kmin, wmax = kmax - kmin;   // window: keys with key - lo <= wmax
-      unsigned krem = (unsigned)k;
-      int bits = 32 - __clz(wmax);
-      for (;;) {
-        const int shift = bits > kLogBins ? bits - kLogBins : 0;
-        for (int b = tid; b < kBins; b += 1024) s_hist[b] = 0;
-        __syncthreads();
-#pragma unroll
-        for (int u = 0; u < kPer; ++u) {
-          const uint32_t d = key[u] - lo;
-          if (u < nm && key[u] >= lo && d <= wmax) atomicAdd(&s_hist[d >> shift], 1u);
-        }
-        __syncthreads();
-        {   // bins in descending order, two per thread
-          const unsigned v0 = s_hist[kBins - 1 - 2 * tid], v1 = s_hist[kBins - 2 - 2 * tid];
-          int tot;
-          const unsigned above = (unsigned)block_excl_scan((int)(v0 + v1), s_scan, tot);
-          if (above < krem && krem <= above + v0) {
-            s_bin = kBins - 1 - 2 * tid; s_krem = krem - above;
-          } else if (above + v0 < krem && krem <= above + v0 + v1) {
-            s_bin = kBins - 2 - 2 * tid; s_krem = krem - above - v0;
-          }
-        }
-        __syncthreads();
-        lo += s_bin << shift;
-        krem = s_krem;
-        __syncthreads();
-        if (shift == 0) break;
-        wmax = (1u << shift) - 1u;
-        bits = shift;
-      }
-      Tk = lo;
-      need = krem;   // entries with key == Tk still to keep, lowest cache index first
-    }
-    // ---- ordered emit: block prefix sums of (greater, equal) counts packed in 64 bits ----
-    unsigned cgt = 0, ceq = 0;
-#pragma unroll
-    for (int u = 0; u < kPer; ++u) {
-      cgt += (u < nm && key[u] > Tk);
-      ceq += (u < nm && key[u] == Tk);
-    }
-    const unsigned long long v = (unsigned long long)cgt | ((unsigned long long)ceq << 32);
-    unsigned long long inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long x = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += x;
-    }
-    if (lane == 31) s_wsum[warp] = inc;
-    __syncthreads();   // also: every thread has read its cache entries
-    if (warp == 0) {
-      const unsigned long long w = s_wsum[lane];
-      unsigned long long winc = w;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned long long x = __shfl_up_sync(0xffffffffu, winc, o);
-        if (lane >= o) winc += x;
-      }
-      s_wsum[lane] = winc - w;
-    }
-    __syncthreads();
-    const unsigned long long excl = s_wsum[warp] + inc - v;
+    // The (B - L)-th largest key and the ordered places: the selection kernel's own routines (one round, the keys in
+    // registers), so that the tie-break rule lives in one place.
+    uint32_t Tk;
+    unsigned need;
+    int nv = nm;
+    sel_kth_key<1024, kPer>(sh, key, nv, 1, [](int) {}, (unsigned)k, Tk, need);
+    unsigned long long total;
+    const unsigned long long excl = sel_counts_before<1024, kPer>(sh, key, nv, Tk, total);   // its barriers: every thread has read its cache entries
     unsigned bgt = (unsigned)(excl & 0xffffffffu), beq = (unsigned)(excl >> 32);
     int32_t *out = kept + (size_t)(t - 1) * k;
 #pragma unroll
     for (int u = 0; u < kPer; ++u) {
       const bool g = u < nm && key[u] > Tk, e = u < nm && key[u] == Tk;
-      if (g || (e && beq < need)) {
-        const int dst = (int)(bgt + min(beq, need));
+      const int dst = sel_place(g, e, bgt, beq, need);
+      if (dst >= 0) {
         cache[dst] = pos[u];
         out[dst] = pos[u];
       }

@@ -68,18 +68,138 @@ __device__ __forceinline__ float key_score(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+// ---- the selection machinery shared by the kernels that keep "the k best keys, ties to the lower index" ----
+// Shared-memory scratch of one CTA of THREADS threads.
+template <int THREADS>
+struct SelShared {
+  unsigned hist[2 * THREADS];
+  int scan[33];
+  unsigned red[64];
+  unsigned bin, krem;
+  unsigned long long wsum[33];
+};
+
+// The k-th largest key T of the keys the CTA holds (0 < k < their number) and how many keys EQUAL to T
+// are still to be kept once every key above T is.  Each thread holds up to PER keys of a round in
+// key[0 .. nv); with several rounds, reload(round) brings a round's keys back (key and nv change).
+// A min/max pass fixes the key window; each histogram pass splits the current window into up to
+// 2 x THREADS equal bins (the bins follow the data, not fixed bit fields, so shared-memory atomics
+// spread out), picks the bin where the count from the top crosses k and narrows the window to it -
+// at most three passes for 32-bit keys.
+template <int THREADS, int PER, class Reload>
+__device__ __forceinline__ void sel_kth_key(SelShared<THREADS> &sh, uint32_t (&key)[PER], int &nv, int rounds,
+                                            Reload reload, unsigned k, uint32_t &T, unsigned &need) {
+  constexpr int kBins = 2 * THREADS, NWARPS = THREADS / 32;
+  constexpr int kLogBins = THREADS == 1024 ? 11 : THREADS == 512 ? 10 : 9;
+  static_assert(THREADS == 1024 || THREADS == 512 || THREADS == 256, "bins = 2 x threads, a power of two");
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
+  for (int round = 0; round < rounds; ++round) {
+    if (rounds > 1) reload(round);
+#pragma unroll
+    for (int j = 0; j < PER; ++j)
+      if (j < nv) { kmin = min(kmin, key[j]); kmax = max(kmax, key[j]); }
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) { sh.red[warp] = kmin; sh.red[32 + warp] = kmax; }
+  __syncthreads();
+  kmin = __reduce_min_sync(0xffffffffu, lane < NWARPS ? sh.red[lane] : 0xffffffffu);
+  kmax = __reduce_max_sync(0xffffffffu, lane < NWARPS ? sh.red[32 + lane] : 0u);
+  T = kmin;
+  need = k;
+  if (kmin == kmax) return;
+  uint32_t lo = kmin, wmax = kmax - kmin;  // window: keys with key - lo <= wmax
+  unsigned krem = k;
+  int bits = 32 - __clz(wmax);
+  for (;;) {
+    const int shift = bits > kLogBins ? bits - kLogBins : 0;
+    for (int b = tid; b < kBins; b += THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    for (int round = 0; round < rounds; ++round) {
+      if (rounds > 1) reload(round);
+#pragma unroll
+      for (int j = 0; j < PER; ++j) {
+        const uint32_t d = key[j] - lo;
+        if (j < nv && key[j] >= lo && d <= wmax) atomicAdd(&sh.hist[d >> shift], 1u);
+      }
+    }
+    __syncthreads();
+    // Bins in descending order, two per thread: the top one is 2 THREADS - 1 - 2 tid.
+    {
+      const unsigned v0 = sh.hist[kBins - 1 - 2 * tid], v1 = sh.hist[kBins - 2 - 2 * tid];
+      int tot;
+      const unsigned above = (unsigned)block_excl_scan((int)(v0 + v1), sh.scan, tot);
+      if (above < krem && krem <= above + v0) {
+        sh.bin = kBins - 1 - 2 * tid; sh.krem = krem - above;
+      } else if (above + v0 < krem && krem <= above + v0 + v1) {
+        sh.bin = kBins - 2 - 2 * tid; sh.krem = krem - above - v0;
+      }
+    }
+    __syncthreads();
+    lo += sh.bin << shift;
+    krem = sh.krem;
+    __syncthreads();
+    if (shift == 0) break;
+    wmax = (1u << shift) - 1u;
+    bits = shift;
+  }
+  T = lo;
+  need = krem;  // keys equal to T still to keep, lowest index first
+}
+
+// How many keys above T (low word) and equal to T (high word) the threads BEFORE this one hold among the
+// keys currently loaded, by one block prefix sum; total = the CTA's counts.  With these, thread order =
+// index order decides which of the tied keys stay: no atomics do.
+template <int THREADS, int PER>
+__device__ __forceinline__ unsigned long long sel_counts_before(SelShared<THREADS> &sh, const uint32_t (&key)[PER], int nv,
+                                                                uint32_t T, unsigned long long &total) {
+  constexpr int NWARPS = THREADS / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned cgt = 0, ceq = 0;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    cgt += (j < nv && key[j] > T);
+    ceq += (j < nv && key[j] == T);
+  }
+  unsigned long long v = (unsigned long long)cgt | ((unsigned long long)ceq << 32), inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();   // the scratch may still be read from the call before
+  if (lane == 31) sh.wsum[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    unsigned long long w = lane < NWARPS ? sh.wsum[lane] : 0ull, winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned long long t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    sh.wsum[lane] = winc - w;
+    if (lane == 31) sh.wsum[32] = winc;
+  }
+  __syncthreads();
+  total = sh.wsum[32];
+  return sh.wsum[warp] + inc - v;
+}
+
+// Place of a key in the kept list given the counts (above T, equal to T) of the keys before it: every key above
+// T is kept, of those equal to T the first `need`; -1 if the key is not kept.
+__device__ __forceinline__ int sel_place(bool greater, bool equal, unsigned bgt, unsigned beq, unsigned need) {
+  if (greater) return (int)(bgt + min(beq, need));
+  if (equal && beq < need) return (int)(bgt + beq);
+  return -1;
+}
+
 template <bool SINGLE, int MODE, int THREADS, int PER>
 __global__ void __launch_bounds__(THREADS) k_select(Ctx c, const float *scores, int32_t *idx, int32_t *kept_count,
                                                          int seg_base, int fill_pages, float *prio,
                                                          const float *noise, int noise_stride, int noise_base) {
-  constexpr int kSelBins = 2 * THREADS, kSelPerThread = PER, kSelRound = THREADS * PER, NWARPS = THREADS / 32;
-  constexpr int kLogBins = THREADS == 1024 ? 11 : THREADS == 512 ? 10 : 9;
-  static_assert(THREADS == 1024 || THREADS == 512 || THREADS == 256, "bins = 2 x threads, a power of two");
-  __shared__ unsigned s_hist[kSelBins];
-  __shared__ int s_scan[33];
-  __shared__ unsigned s_red[64];
-  __shared__ unsigned s_bin, s_krem;
-  __shared__ unsigned long long s_wsum[33];
+  constexpr int kSelPerThread = PER, kSelRound = THREADS * PER;
+  __shared__ SelShared<THREADS> sh;
   if ((int)blockIdx.x >= c.planhdr[PH_NWORK]) return;
   const int seg = c.work[blockIdx.x];
   const SegPlan p = c.plan[seg];
@@ -128,105 +248,26 @@ __global__ void __launch_bounds__(THREADS) k_select(Ctx c, const float *scores, 
   };
   if (SINGLE) load_round(0);
 
-  // ---- key window ----
-  uint32_t kmin = 0xffffffffu, kmax = 0u;
-  for (int round = 0; round < rounds; ++round) {
-    if (!SINGLE) load_round(round);
-#pragma unroll
-    for (int j = 0; j < kSelPerThread; ++j)
-      if (j < nv) { kmin = min(kmin, key[j]); kmax = max(kmax, key[j]); }
-  }
-  kmin = __reduce_min_sync(0xffffffffu, kmin);
-  kmax = __reduce_max_sync(0xffffffffu, kmax);
-  if (lane == 0) { s_red[warp] = kmin; s_red[32 + warp] = kmax; }
-  __syncthreads();
-  kmin = __reduce_min_sync(0xffffffffu, lane < NWARPS ? s_red[lane] : 0xffffffffu);
-  kmax = __reduce_max_sync(0xffffffffu, lane < NWARPS ? s_red[32 + lane] : 0u);
-
-  uint32_t T = kmin;
-  unsigned need = (unsigned)k;
-  if (kmin != kmax) {
-    uint32_t lo = kmin, wmax = kmax - kmin;  // window: keys with key - lo <= wmax
-    unsigned krem = (unsigned)k;
-    int bits = 32 - __clz(wmax);
-    for (;;) {
-      const int shift = bits > kLogBins ? bits - kLogBins : 0;
-      for (int b = tid; b < kSelBins; b += THREADS) s_hist[b] = 0;
-      __syncthreads();
-      for (int round = 0; round < rounds; ++round) {
-        if (!SINGLE) load_round(round);
-#pragma unroll
-        for (int j = 0; j < kSelPerThread; ++j) {
-          const uint32_t d = key[j] - lo;
-          if (j < nv && key[j] >= lo && d <= wmax) atomicAdd(&s_hist[d >> shift], 1u);
-        }
-      }
-      __syncthreads();
-      // Bins in descending order, two per thread: 2047 - 2 tid, then 2046 - 2 tid.
-      {
-        const unsigned v0 = s_hist[kSelBins - 1 - 2 * tid], v1 = s_hist[kSelBins - 2 - 2 * tid];
-        int tot;
-        const unsigned above = (unsigned)block_excl_scan((int)(v0 + v1), s_scan, tot);
-        if (above < krem && krem <= above + v0) {
-          s_bin = kSelBins - 1 - 2 * tid; s_krem = krem - above;
-        } else if (above + v0 < krem && krem <= above + v0 + v1) {
-          s_bin = kSelBins - 2 - 2 * tid; s_krem = krem - above - v0;
-        }
-      }
-      __syncthreads();
-      lo += s_bin << shift;
-      krem = s_krem;
-      __syncthreads();
-      if (shift == 0) break;
-      wmax = (1u << shift) - 1u;
-      bits = shift;
-    }
-    T = lo;
-    need = krem;  // pairs with key == T still to keep, lowest slots first
-  }
+  uint32_t T;
+  unsigned need;
+  sel_kth_key<THREADS, PER>(sh, key, nv, rounds, load_round, (unsigned)k, T, need);
 
   // ---- ordered emit: one block prefix sum per round ----
   unsigned run_gt = 0, run_eq = 0;
   for (int round = 0; round < rounds; ++round) {
     if (!SINGLE) load_round(round);
-    unsigned cgt = 0, ceq = 0;
-#pragma unroll
-    for (int j = 0; j < kSelPerThread; ++j) {
-      cgt += (j < nv && key[j] > T);
-      ceq += (j < nv && key[j] == T);
-    }
-    // Exclusive block scan of (cgt, ceq) packed in 64 bits.
-    unsigned long long v = (unsigned long long)cgt | ((unsigned long long)ceq << 32), inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
-    }
-    __syncthreads();
-    if (lane == 31) s_wsum[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-      unsigned long long w = lane < NWARPS ? s_wsum[lane] : 0ull, winc = w;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        unsigned long long t = __shfl_up_sync(0xffffffffu, winc, o);
-        if (lane >= o) winc += t;
-      }
-      s_wsum[lane] = winc - w;
-      if (lane == 31) s_wsum[32] = winc;
-    }
-    __syncthreads();
-    const unsigned long long excl = s_wsum[warp] + inc - v, tot = s_wsum[32];
+    unsigned long long tot;
+    const unsigned long long excl = sel_counts_before<THREADS, PER>(sh, key, nv, T, tot);
     unsigned bgt = run_gt + (unsigned)(excl & 0xffffffffu), beq = run_eq + (unsigned)(excl >> 32);
     const int slot0 = round * kSelRound + tid * kSelPerThread;
 #pragma unroll
     for (int j = 0; j < kSelPerThread; ++j) {
       const bool g = j < nv && key[j] > T, e = j < nv && key[j] == T;
+      const int dst = sel_place(g, e, bgt, beq, need);
       if (MODE == 0) {
-        if (g) out[bgt + min(beq, need)] = slot0 + j;
-        else if (e && beq < need) out[bgt + beq] = slot0 + j;
+        if (dst >= 0) out[dst] = slot0 + j;
       } else if (j < nv) {
-        const bool kept = g || (e && beq < need);
+        const bool kept = dst >= 0;
         const int rank = slot0 + j - (int)(bgt + min(beq, need));   // candidates before this slot
         pr[slot0 + j] = kept ? INFINITY : key_score(key[j]) - nz[rank];
       }
