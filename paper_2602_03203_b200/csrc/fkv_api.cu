@@ -338,13 +338,18 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
     const int n = c->h_len[(size_t)layer * batch + s] + ((app && seq_mask.has(s)) ? 1 : 0);
     maxpages = std::max(maxpages, (n + kPage - 1) / kPage);
   }
-  // Splits per segment: CTAs for about three quarters of the SMs per launch, at least kAttendMinPages pages each.
-  // Consecutive launches of a decode step share the SMs (three CTAs fit on one); a launch on its own gains
-  // nothing from more CTAs either - the merge in the segment's last CTA grows with the splits (measured: 17 us
-  // per layer launch at 14 splits, 17.6 at 20, 20.4 at 32 on 8 segments of 8192 pairs).
+  // Splits per segment, at least kAttendMinPages pages each.  Consecutive launches of a decode step share the SMs
+  // (three CTAs fit on one): CTAs for about three quarters of the SMs per launch.  A launch on its own has the GPU to
+  // itself and lasts as long as its longest CTA: CTAs for every slot of every SM - but never more than
+  // kSoloMaxSplits per segment, because the merge in a segment's last CTA grows with the splits (8 segments of 8192
+  // pairs: 16.9 us per layer launch at 14 splits, 17.6 at 20, 20.4 at 32; 64 segments of 2K - 16K pairs: 96 us at 2
+  // splits, which this rule turns into 7).
+  constexpr int kSoloMaxSplits = 14;
   const int nseg = batch * Hkv;
-  const int want_ctas = c->sm_count * 3 / 4;
-  int splits = std::min(c->lay.att_smax, std::max(1, (want_ctas + nseg / 2) / nseg));
+  const int want_ctas = pdl ? c->sm_count * 3 / 4 : c->sm_count * 3;
+  // (a launch on its own must fit one wave: rounded down, so that no CTA starts after the others have finished)
+  int splits = std::min(c->lay.att_smax, std::max(1, pdl ? (want_ctas + nseg / 2) / nseg : want_ctas / nseg));
+  if (!pdl) splits = std::min(splits, kSoloMaxSplits);
   splits = std::max(1, std::min(splits, maxpages / kAttendMinPages));
   const int pps = std::max(1, (maxpages + splits - 1) / splits);
   if (scale == 0.f) scale = 1.f / sqrtf((float)D);

@@ -160,6 +160,7 @@ __global__ void __launch_bounds__(NCW * 32, 1) k_score(Ctx c, float *out, int se
   PageWalk cur = {wi0, 0, 0, 0, 0, 0};
   int scorer = -1, seg_held = -1;    // (layer, head) whose weights the warp holds; the segment last seen
   int slot_i = warp, ph = 0;         // ring slot of page v and the parity of its barrier's current phase
+  bool gave_up = false;
   for (int v = warp; walk_to(c, cur, v, t0, t1, nwork, NCW); v += NCW) {
     // The page that will take this slot next: looked up now, copied when this page has been scored.
     const int pid_next = walk_to(c, ahead, v + nslots, t0, t1, nwork, NCW)
@@ -188,7 +189,7 @@ __global__ void __launch_bounds__(NCW * 32, 1) k_score(Ctx c, float *out, int se
       __syncwarp();
       }
     }
-    if (!mbar_wait(smem_u32(&bars[slot_i]), ph)) { set_status(c, kDevWaitTimeout); break; }
+    if (!mbar_wait(smem_u32(&bars[slot_i]), ph)) { set_status(c, kDevWaitTimeout); gave_up = true; break; }
     const uint8_t *page = smem + (size_t)slot_i * pitch;
     const uint32_t kbase = smem_u32(page), vbase = kbase + c.off_v;
     // Eight accumulators (four chains for each half of the hidden units), summed below in a fixed order, so that
@@ -258,6 +259,14 @@ __global__ void __launch_bounds__(NCW * 32, 1) k_score(Ctx c, float *out, int se
     slot_i += NCW;
     if (slot_i >= nslots) { slot_i -= nslots; ph ^= 1; }
   }
+  // After a wait that ran out the warp leaves early: give the copies it still has in flight (the pages it would
+  // have scored next) one more bounded wait each, so that none lands in shared memory the CTA has given up.
+  if (gave_up)
+    for (int j = 1; j < nslots / NCW; ++j) {
+      slot_i += NCW;
+      if (slot_i >= nslots) { slot_i -= nslots; ph ^= 1; }
+      mbar_wait(smem_u32(&bars[slot_i]), ph);
+    }
 }
 
 // Baseline scores that need no learned scorer (Appendix E.2): one attention-feature column averaged
