@@ -94,6 +94,24 @@ def test_score_parity(cfg):
     assert ld.cache.device_status()[0] == 0
 
 
+@pytest.mark.parametrize("g,D", [(1, 64), (2, 128), (3, 64), (5, 128), (6, 64), (8, 128), (8, 64)])
+def test_score_group_sizes_and_head_dims(g, D):
+    # Feature widths 6g that are and are not multiples of the 8-column tf32 steps (the column after the last
+    # feature is the position id and must never be read as one), both head dimensions, ring sizes that follow
+    # from the page size; three segments of different lengths so that every CTA crosses segment boundaries.
+    w = wl.Workload("gd", 1, 3, g, D, (700, 33, 1234), (1 << 20,) * 3, 0, 61, "channel_lognormal")
+    ld = Loaded(w)
+    got = npf(ld.cache.score(0))
+    worst = 0.0
+    for s, n in enumerate(w.lens):
+        for h in range(w.num_kv_heads):
+            K, V, A, _ = ld.head(0, s, h)
+            ref = oracle.score(K, V, A, *ld.weights(0, h))
+            worst = max(worst, float(np.abs(got[s, h, :n] - ref).max()))
+    assert worst <= SCORE_TOL, worst
+    assert ld.cache.device_status()[0] == 0
+
+
 @pytest.mark.parametrize("act", [binding.ACT_SILU, binding.ACT_GELU_TANH, binding.ACT_SIGMOID])
 def test_score_other_activations(act):
     w = dataclasses.replace(small(1), activation=act)
