@@ -105,3 +105,26 @@ def test_rkv_one_layer_of_the_32k_configuration():
         ref = oracle.score_rkv(Kb[h], Ab[h], w.group_size, rows=rows)
         assert np.abs(got[0, h, rows] - ref).max() <= SCORE_TOL
     assert c.device_status()[0] == 0
+
+
+def test_rkv_with_an_empty_sequence_and_per_sequence_budgets():
+    # Three sequence slots, the middle one never filled; the other two with their own budgets.
+    w = wl.Workload("rkv_e", 1, 2, 4, 128, (400, 300, 650), (1 << 20, 1 << 20, 1 << 20), 16, 53, "normal")
+    c = binding.from_workload(w)
+    host = {}
+    for s in (0, 2):
+        K, V, A, pos = wl.layer_inputs(w, 0, s)
+        c.prefill(0, s, K.cuda(), V.cuda(), A.cuda(), pos.cuda())
+        host[s] = (bits(K), npf(A), npf(pos))
+    c.set_budget(0, 100); c.set_budget(2, 333)
+    sc = npf(c.score_rkv(0))
+    c.evict_rkv(0)
+    assert c.lengths(0) == [100, 0, 333]
+    for s, B in ((0, 100), (2, 333)):
+        Kb, A, pos = host[s]
+        n = w.lens[s]
+        for h in range(2):
+            assert np.abs(sc[s, h, :n] - oracle.score_rkv(Kb[h], A[h], 4)).max() <= SCORE_TOL
+            _, _, _, p2 = c.export_head(0, s, h)
+            assert np.array_equal(npf(p2), pos[oracle.select(sc[s, h, :n], B, 16)])
+    assert c.device_status()[0] == 0
