@@ -148,6 +148,7 @@ struct fkv_cache {
   std::vector<uint8_t> staging;
   uint64_t launches = 0;
   int sm_count = 148;
+  int max_cluster = 0;        // largest attention cluster the device places (found at the first stand-alone launch)
   float feature_scale = 0.f;  // softmax scale of the recorded queries (the last decode call's)
   bool timing = false, timed = false;
   cudaEvent_t ev[7] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};  // [6]: after the plan
@@ -301,11 +302,12 @@ int launch_compact(fkv_cache *c, const int32_t *idx, int seg_base, int max_new, 
 }
 
 // One launch of the attention kernel: `splits` CTAs per segment.  pdl: the launch may run alongside the one
-// before it on the stream.
-template <int D, int NCW, int SLOTS>
+// before it on the stream.  cluster: the splits of a segment are one thread-block cluster (the merge goes through
+// distributed shared memory).
+template <int D, int NCW, int SLOTS, bool CLUSTER>
 int launch_attend_t(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cudaStream_t st) {
-  const size_t smem = AttendSmem::bytes(D, NCW, SLOTS);
-  auto kern = k_attend<D, NCW, SLOTS>;
+  const size_t smem = AttendSmem::bytes(D, NCW, SLOTS, CLUSTER);
+  auto kern = k_attend<D, NCW, SLOTS, CLUSTER>;
   static SmemOptIn opt_in;
   FKV_CUDA(opt_in.ensure(kern, smem));
   cudaLaunchConfig_t cfg = {};
@@ -313,19 +315,57 @@ int launch_attend_t(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cud
   cfg.blockDim = dim3((NCW + 1) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (pdl || a->wait_first) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (CLUSTER) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = splits; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+    ++na;
+  }
   cfg.attrs = at;
-  cfg.numAttrs = (pdl || a->wait_first) ? 1 : 0;
+  cfg.numAttrs = na;
   FKV_CUDA(cudaLaunchKernelEx(&cfg, kern, c->ctx, *a));
   ++c->launches;
   return FKV_OK;
 }
 
-int attend_dispatch(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, cudaStream_t st) {
-  return c->cfg.head_dim == 128 ? launch_attend_t<128, 4, 8>(c, a, splits, pdl, st)
-                                : launch_attend_t<64, 4, 16>(c, a, splits, pdl, st);
+// The largest cluster of attention CTAs this device places: 16 (needs the non-portable opt-in), else 8; found once
+// per handle.
+template <int D, int NCW, int SLOTS>
+int attend_max_cluster(fkv_cache *c) {
+  auto kern = k_attend<D, NCW, SLOTS, true>;
+  const size_t smem = AttendSmem::bytes(D, NCW, SLOTS, true);
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+      cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 1;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kClusterSplits, 1);
+  cfg.blockDim = dim3((NCW + 1) * 32);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = kClusterSplits; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  int nclusters = 0;
+  const bool ok16 = cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg) == cudaSuccess && nclusters > 0;
+  (void)cudaGetLastError();
+  return ok16 ? kClusterSplits : 8;
+}
+
+int attend_dispatch(fkv_cache *c, const AttendArgs *a, int splits, bool pdl, bool cluster, cudaStream_t st) {
+  if (cluster)
+    return c->cfg.head_dim == 128 ? launch_attend_t<128, 4, 8, true>(c, a, splits, pdl, st)
+                                  : launch_attend_t<64, 4, 16, true>(c, a, splits, pdl, st);
+  return c->cfg.head_dim == 128 ? launch_attend_t<128, 4, 8, false>(c, a, splits, pdl, st)
+                                : launch_attend_t<64, 4, 16, false>(c, a, splits, pdl, st);
 }
 
 // Attention over `layer`, with the new pair of every participating sequence appended first when k_new is given.
@@ -351,6 +391,17 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
   int splits = std::min(c->lay.att_smax, std::max(1, pdl ? (want_ctas + nseg / 2) / nseg : want_ctas / nseg));
   if (!pdl) splits = std::min(splits, kSoloMaxSplits);
   splits = std::max(1, std::min(splits, maxpages / kAttendMinPages));
+  // A launch on its own over few segments: the splits of a segment as one cluster of 16 (or 8) CTAs, merged through
+  // distributed shared memory.  The cluster size is a power of two; with many segments the global-memory merge
+  // above, whose split count is free, fills the GPU better.
+  bool cluster = false;
+  if (!pdl && nseg * kClusterSplits <= c->sm_count * 3 / 2) {
+    if (c->max_cluster == 0)
+      c->max_cluster = c->cfg.head_dim == 128 ? attend_max_cluster<128, 4, 8>(c) : attend_max_cluster<64, 4, 16>(c);
+    int cs = 1;
+    while (cs * 2 <= c->max_cluster && cs * 2 <= kClusterSplits && maxpages / (cs * 2) >= kAttendMinPages) cs *= 2;
+    if (cs >= 8) { cluster = true; splits = cs; }
+  }
   const int pps = std::max(1, (maxpages + splits - 1) / splits);
   if (scale == 0.f) scale = 1.f / sqrtf((float)D);
   if (app) c->feature_scale = scale;
@@ -359,7 +410,7 @@ int launch_attend(fkv_cache *c, int layer, const void *q, void *out, float scale
   a.scale_log2 = scale * 1.4426950408889634f; a.pps = pps; a.append = app ? 1 : 0;
   a.k_new = (const uint8_t *)k_new; a.v_new = (const uint8_t *)v_new; a.pos_new = pos; a.seq_mask = seq_mask;
   a.wait_first = pdl ? 0 : 1;
-  const int rc = attend_dispatch(c, &a, splits, pdl, st);
+  const int rc = attend_dispatch(c, &a, splits, pdl, cluster, st);
   if (rc) return rc;
   if (app)
     for (int s = 0; s < batch; ++s)

@@ -51,6 +51,7 @@
 namespace fkv {
 
 constexpr int kMaxSplits = 32;   // splits per segment (one lane of the merging warp per split)
+constexpr int kClusterSplits = 16;   // splits per segment when they form one thread-block cluster
 
 struct AttendSmem {
   // ring | slot barriers (512 B)
@@ -59,7 +60,12 @@ struct AttendSmem {
     const size_t r = (size_t)slots * (4 * D * kPage), merge = (size_t)ncw * 8 * (D + 4) * 4;
     return ((r > merge ? r : merge) + 127) & ~(size_t)127;
   }
-  static __host__ __device__ size_t bytes(int D, int ncw, int slots) { return ring(D, ncw, slots) + kBars; }
+  // With the cluster merge: this CTA's slice of the output from every split (8 query rows x D floats in all) and
+  // every split's statistics (16 splits x 8 rows x (m, l)).
+  static __host__ __device__ size_t recv(int D) { return (size_t)8 * D * 4 + (size_t)kClusterSplits * 8 * 8; }
+  static __host__ __device__ size_t bytes(int D, int ncw, int slots, bool cluster = false) {
+    return ring(D, ncw, slots) + kBars + (cluster ? recv(D) : 0);
+  }
 };
 
 struct AttendArgs {
@@ -80,6 +86,23 @@ struct AttendArgs {
 __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 0;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// All threads of all CTAs of the cluster: writes made before (also into other CTAs' shared memory) are visible after.
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of this CTA's shared-memory location `local` in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void dsmem_st4(uint32_t addr, float4 v) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+               : "memory");
+}
+__device__ __forceinline__ void dsmem_st2(uint32_t addr, float x, float y) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(x), "f"(y) : "memory");
+}
 // The merge of a segment's split partials, run by the whole CTA that finished last.  part: [nact][G][D + 4] fp32
 // (O relative to the partial's own maximum, then m and l); out: G rows of D bf16; scratch: shared memory,
 // NW * 8 * D + 16 floats.  One round trip to L2 per pass: warp w asks for partials w, w + NW, ... (PASS of them
@@ -173,7 +196,12 @@ __device__ __forceinline__ void merge_partials(const float *part, int nact, int 
   }
 }
 
-template <int D, int NCW, int SLOTS>
+// CLUSTER: the splits of a segment (the grid's x extent, a power of two <= kClusterSplits) are one thread-block
+// cluster and merge through distributed shared memory instead of global memory: every CTA owns a slice of the
+// segment's output, receives that slice of every split's partial, and after one cluster barrier reduces and writes
+// it - no partial leaves the SMs and no ticket is taken.  For launches that run on their own (the per-layer entry
+// points at small batch), where the merge's round trips to L2 are a sixth of the launch.
+template <int D, int NCW, int SLOTS, bool CLUSTER>
 __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx c, AttendArgs a) {
   constexpr int KSQ = D / 16;  // k-steps of K Q^T
   constexpr int MT = D / 16;   // m-tiles (16 channels) of O^T = V^T P^T
@@ -196,6 +224,9 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   // (Asking the pages into L2 ahead of the wait was measured and set aside: the early traffic slows the kernel
   // that is still running by more than it saves this one.)
   if (a.wait_first) griddep_wait();
+  // Cluster merge: every CTA says "I am running" now and checks, just before it writes into the others' shared
+  // memory, that all of them have said so.
+  if (CLUSTER && S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   int *ptrow = c.pt + (size_t)seg * c.max_pages;
   // The producer warp asks for its first page-table entries before the length is known, at the place the host's
   // pages-per-split figure puts them (entries past the segment's pages are never used), so that the two reads
@@ -435,7 +466,101 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
   }
   __syncthreads();
 
-  if (S == 1) {
+  if (CLUSTER && S > 1) {
+    float *recv_o = reinterpret_cast<float *>(smem + ring_bytes + AttendSmem::kBars);   // [S][per]: my slice of every split's O
+    float *recv_ml = recv_o + 8 * D;                                                     // [S][8][2]: every split's (m, l)
+    // ---- push: elements [o * per, (o + 1) * per) of this CTA's merged partial go to CTA o of the cluster (its
+    // slot `rank`), four channels per store; the producer warp sends the (m, l) of every query row to every CTA ----
+    const int per = G * D / S;   // output elements per owner: S is a power of two <= 16 and 64 divides G * D
+    const uint32_t recv_o_s = smem_u32(recv_o), recv_ml_s = smem_u32(recv_ml);
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every CTA of the cluster has started
+    if (warp < NCW) {
+      for (int e = tid * 4; e < G * D; e += NCW * 32 * 4) {
+        const int r = e / D, ch = e - r * D;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (active) {
+          float mw[NCW], M = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) {
+            mw[w] = mg[((size_t)w * 8 + r) * MGS + D];
+            M = fmaxf(M, mw[w]);
+          }
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) {
+            const float f = mw[w] == -INFINITY ? 0.f : exp2f(mw[w] - M);
+            const float4 x = *reinterpret_cast<const float4 *>(mg + ((size_t)w * 8 + r) * MGS + ch);
+            acc.x = fmaf(f, x.x, acc.x); acc.y = fmaf(f, x.y, acc.y);
+            acc.z = fmaf(f, x.z, acc.z); acc.w = fmaf(f, x.w, acc.w);
+          }
+        }
+        const int owner = e / per;
+        dsmem_st4(dsmem_addr(recv_o_s + (uint32_t)(rank * per + (e - owner * per)) * 4u, owner), acc);
+      }
+    } else {
+      for (int e = lane; e < S * G; e += 32) {
+        const int owner = e / G, r = e - owner * G;
+        float M = -INFINITY, l = 0.f;
+        if (active) {
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) M = fmaxf(M, mg[((size_t)w * 8 + r) * MGS + D]);
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) {
+            const float *rw = mg + ((size_t)w * 8 + r) * MGS;
+            l += (rw[D] == -INFINITY ? 0.f : exp2f(rw[D] - M)) * rw[D + 1];
+          }
+        }
+        dsmem_st2(dsmem_addr(recv_ml_s + (uint32_t)(rank * 8 + r) * 8u, owner), M, l);
+      }
+    }
+    cluster_sync_all();
+    // ---- reduce the slice this CTA owns, [rank * per, (rank + 1) * per), over the S partials and write it: one
+    // warp per query row of the slice; lane s holds the statistics of partial s; the lanes form 4 groups that each
+    // sum every fourth partial for 8 x 4 channels, and the groups are added with shuffles ----
+    const int lo = rank * per, hi = lo + per;
+    for (int r = lo / D + warp; r * D < hi; r += NCW + 1) {
+      const int e0 = max(lo, r * D), e1 = min(hi, (r + 1) * D);
+      const float ms = lane < S ? recv_ml[(lane * 8 + r) * 2] : -INFINITY;
+      const float ls = lane < S ? recv_ml[(lane * 8 + r) * 2 + 1] : 0.f;
+      float M = ms;
+#pragma unroll
+      for (int sh = 16; sh >= 1; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
+      const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
+      float L = f * ls;
+#pragma unroll
+      for (int sh = 16; sh >= 1; sh >>= 1) L += __shfl_xor_sync(0xffffffffu, L, sh);
+      const float inv = L > 0.f ? 1.f / L : 0.f;   // an empty sequence gives zeros
+      const int grp = lane >> 3, l8 = lane & 7;
+      for (int base = e0; base < e1; base += 32) {
+        const int e = base + l8 * 4;
+        const bool valid = e < e1;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < kClusterSplits / 4; ++k) {
+          const int sp = grp + 4 * k;
+          const float fs = __shfl_sync(0xffffffffu, f, sp);
+          if (sp < S && valid) {
+            const float4 x = *reinterpret_cast<const float4 *>(recv_o + sp * per + (e - lo));
+            acc.x = fmaf(fs, x.x, acc.x); acc.y = fmaf(fs, x.y, acc.y);
+            acc.z = fmaf(fs, x.z, acc.z); acc.w = fmaf(fs, x.w, acc.w);
+          }
+        }
+#pragma unroll
+        for (int sh = 8; sh <= 16; sh <<= 1) {
+          acc.x += __shfl_xor_sync(0xffffffffu, acc.x, sh); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, sh);
+          acc.z += __shfl_xor_sync(0xffffffffu, acc.z, sh); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, sh);
+        }
+        if (grp == 0 && valid) {
+          const __nv_bfloat162 p0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+          const __nv_bfloat162 p1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+          uint2 pk;
+          pk.x = *reinterpret_cast<const uint32_t *>(&p0);
+          pk.y = *reinterpret_cast<const uint32_t *>(&p1);
+          *reinterpret_cast<uint2 *>(a.out + qrow0 * D + e) = pk;
+        }
+      }
+      if (rec && e0 == r * D && lane == 0) hist_mp[(size_t)r * c.hist_wp] = M + log2f(L);
+    }
+  } else if (S == 1) {
     // ---- one CTA holds the whole segment (many segments per launch, or a short one): normalise and write the
     // output straight from the warps' partials; nothing goes through global memory and no ticket is taken ----
     if (warp < NCW) {

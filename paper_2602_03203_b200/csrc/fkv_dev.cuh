@@ -82,7 +82,11 @@ constexpr int kMaxBatch = 256;
 struct SeqMask {
   unsigned long long w[kMaxBatch / 64];
   int use;
-  __host__ __device__ bool has(int s) const { return !use || ((w[s >> 6] >> (s & 63)) & 1ull); }
+  __host__ __device__ bool has(int s) const {   // (no indexed access: the struct is a kernel parameter)
+    const unsigned long long x = s < 64 ? w[0] : s < 128 ? w[1] : s < 192 ? w[2] : w[3];
+    return !use || ((x >> (s & 63)) & 1ull);
+  }
+  static_assert(kMaxBatch == 256, "four words");
 };
 
 __device__ __forceinline__ int seg_of(const Ctx &c, int layer, int seq, int head) {
