@@ -303,6 +303,29 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
     cta_sync();                       // the barriers are set up
   }
 
+  // ---- the length grows once every CTA of the sequence (all heads, all splits) has read the old one: a ticket per
+  // CTA, taken by the producer warp's first lane as soon as the CTA's part of the append is done (early in the
+  // kernel, so that the atomic's round trip is not on the way out); the last ticket moves the length ----
+  auto take_length_ticket = [&]() {
+    const int total = (int)gridDim.x * c.Hkv, ls = a.layer * c.batch + seq;
+    int *ticket = &c.seq_tickets[ls];
+    __threadfence();   // this CTA's page-table and failure writes come before its ticket
+    const int tk = atomicAdd(ticket, 1);
+    if (tk == total - 1) {
+      *ticket = 0;
+      __threadfence();
+      if ((n_old % kPage) == 0 && atomicExch(&c.seq_fail[ls], 0) != 0) {
+        // a head found no free page: no head's length moves, the token is not recorded
+      } else {
+        c.len[ls] = n_old + 1;
+        if (rec) {
+          c.hist_n[(size_t)ls * c.hist_w + hcnt % c.hist_w] = n_old + 1;
+          c.hist_cnt[ls] = hcnt + 1;
+        }
+      }
+    }
+  };
+
   if (active && warp == NCW) {
     if (tail) {
       // The new pair goes to slot n_old of the page record (and, below, into the consumer's copy of the page).
@@ -340,6 +363,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
       }
       __syncwarp();
     }
+    if (app && lane == 0) take_length_ticket();
+    __syncwarp();
     // The pages that did not fit the empty ring, in page order and NCW at a time (one page of every consumer warp:
     // their slots come free together).  The whole warp waits, converged, for the previous pages of the group's
     // slots to be consumed; then lanes 0 .. NCW-1 issue one copy each.
@@ -359,6 +384,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
       }
       if (lane < NCW && i + lane < npg) issue(i + lane, pid);
     }
+  } else if (warp == NCW) {
+    if (app && lane == 0) take_length_ticket();   // a CTA without pages still counts
   } else if (active) {
     // ---------------- consumers: warp w takes pages w, w + NCW, ... of this CTA ----------------
     // Q^T as B fragments (channels x queries): column gid = query head gid of the group (zero beyond g).
@@ -660,26 +687,6 @@ __global__ void __launch_bounds__((NCW + 1) * 32, NCW <= 4 ? 3 : 1) k_attend(Ctx
           __ldcg(reinterpret_cast<const uint4 *>(a.q + qrow0 * D) + i);
     }
 
-  // ---- the length grows once every CTA of the sequence (all heads, all splits) has read the old one ----
-  if (app && tid == 0) {
-    const int total = (int)gridDim.x * c.Hkv, ls = a.layer * c.batch + seq;
-    int *ticket = &c.seq_tickets[ls];
-    __threadfence();   // this CTA's page-table and failure writes come before its ticket
-    const int tk = atomicAdd(ticket, 1);
-    if (tk == total - 1) {
-      *ticket = 0;
-      __threadfence();
-      if ((n_old % kPage) == 0 && atomicExch(&c.seq_fail[ls], 0) != 0) {
-        // a head found no free page: no head's length moves, the token is not recorded
-      } else {
-        c.len[ls] = n_old + 1;
-        if (rec) {
-          c.hist_n[(size_t)ls * c.hist_w + hcnt % c.hist_w] = n_old + 1;
-          c.hist_cnt[ls] = hcnt + 1;
-        }
-      }
-    }
-  }
   // A launch with the programmatic attribute starts without waiting for the launch before it; it must not be
   // COMPLETE before that one is, or whatever is ordered after this grid (the next decode step, an eviction, the end
   // of a recorded graph) would not be ordered after the whole chain.  One thread of the grid waits for the

@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(1024) k_golden_select(const float *alpha, int 
   constexpr int kPer = 8;
   __shared__ SelShared<1024> sh;
   int *cache = reinterpret_cast<int *>(gsm);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   const int per = (B + 1023) / 1024, j0 = min(B, tid * per), j1 = min(B, j0 + per), nm = j1 - j0;
   const int k = B - L;
   for (int j = tid; j < B; j += 1024) cache[j] = j;

@@ -203,7 +203,7 @@ __global__ void __launch_bounds__(THREADS) k_select(Ctx c, const float *scores, 
   if ((int)blockIdx.x >= c.planhdr[PH_NWORK]) return;
   const int seg = c.work[blockIdx.x];
   const SegPlan p = c.plan[seg];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   if (fill_pages) fill_pt_new(c, seg, p);
   const int m = p.n_old - p.r;
   const int k = MODE == 0 ? p.k_sel : max(0, m - 2 * (p.n_old - p.n_new));   // MODE 1: the non-candidates
