@@ -3,7 +3,7 @@
 The score's similarity term is the n x n contraction of a segment's keys on the tensor cores; the
 cases span one pair, lengths around the 128-row operand tiles and the 256-row units, ragged last
 tiles, several segments of different lengths per launch, both head dimensions, duplicate and zero
-keys.  Tolerance: 1e-3 on the scores (the benchmark spec's figure for scores); selection and
+keys.  Tolerance: 1e-3 on the scores (the figure every score of this library is held to); selection and
 compaction from the GPU's own scores are bit-exact.
 """
 import numpy as np
