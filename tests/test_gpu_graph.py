@@ -156,3 +156,45 @@ def test_overlapped_decode_steps_are_reproducible_at_full_occupancy():
             ref, ref64 = oracle.attend(qb[t, l, 0, h * g:(h + 1) * g], k2[:n], v2[:n])
             err = np.abs(bits_to_f64(ob[t, l, 0, h * g:(h + 1) * g]) - bits_to_f64(ref))
             assert (err <= np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64))).all(), (l, h, t, err.max())
+
+
+@pytest.mark.parametrize("lens,Hkv", [((3000,), 2), ((700, 5000), 1)])
+def test_replayed_per_layer_calls_match_ordinary_calls(lens, Hkv):
+    """The per-layer entry point (fkv_append_decode_attn) recorded layer by layer and replayed.  At these sizes its
+    launches are the ones whose splits form a thread-block cluster and merge through distributed shared memory; every
+    replay is compared with the same calls made directly on a second cache, and the last one with the oracle."""
+    L, steps = 3, 40
+    w = wl.Workload("graph_layer", L, Hkv, 4, 128, lens, (1 << 20,) * len(lens), 0, 27, "channel_lognormal")
+    a = Loaded(w, max_tokens=max(lens) + steps + 8)
+    b = Loaded(w, max_tokens=max(lens) + steps + 8)
+    ks, vs, qs = _static_inputs(w, L)
+    out_g = torch.zeros_like(qs)
+    a.cache.append_decode_attn(0, ks[0], vs[0], qs[0], out_g[0])   # first launches (set-up) before the capture
+    b.cache.append_decode_attn(0, ks[0], vs[0], qs[0])
+    torch.cuda.synchronize()
+    snap = a.cache.snapshot()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for l in range(L):
+            a.cache.append_decode_attn(l, ks[l], vs[l], qs[l], out_g[l])
+    torch.cuda.synchronize()
+    a.cache.restore(snap)
+    for step in range(steps):
+        graph.replay()
+        out_e = torch.stack([b.cache.append_decode_attn(l, ks[l], vs[l], qs[l]) for l in range(L)])
+        torch.cuda.synchronize()
+        assert torch.equal(out_g, out_e), step          # same launches, same splits: the same bits
+    a.cache.sync_lengths()
+    for l in range(L):
+        assert a.cache.lengths(l) == b.cache.lengths(l)
+    og, qb, g = bits(out_g), bits(qs), w.group_size
+    for l in range(L):
+        for s in range(w.batch):
+            for h in range(Hkv):
+                ka, va, _, _ = a.export(l, s, h)
+                ref, ref64 = oracle.attend(qb[l, s, h * g:(h + 1) * g], ka, va)
+                err = np.abs(bits_to_f64(og[l, s, h * g:(h + 1) * g]) - bits_to_f64(ref))
+                assert np.all(err <= np.maximum(ATTN_TOL, 2.0 ** -7 * np.abs(ref64)))
+    assert a.cache.device_status()[0] == 0 and b.cache.device_status()[0] == 0
