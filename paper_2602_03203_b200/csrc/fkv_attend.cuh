@@ -22,13 +22,20 @@
 //     round trip to L2, every load in flight at once) and writes the output.
 //     A CTA that is not last exits as soon as its partial is out, so its
 //     shared memory is free for the next launch.
+//   - A launch that runs on its own over few segments (the per-layer entry
+//     points at small batch) merges differently: the splits of a segment are
+//     one thread-block cluster, every CTA owns a slice of the output and
+//     receives that slice of every split's partial in its shared memory
+//     (distributed shared memory stores), and after one cluster barrier each
+//     CTA reduces and writes its slice.  No partial touches L2.
 //
 // The launch can also APPEND the token's new (k, v) pair first (Section 3.1:
 // the cache grows by one pair per generated token): the CTA whose page range
 // holds slot n writes the row into the page record and patches its own
 // shared-memory copy of that page, so the pair is attended in the same launch
-// and a decode step is one launch per layer.  The length is bumped by the last
-// CTA of the sequence to finish (an atomic ticket), after every CTA has read it.
+// and a decode step is one launch per layer.  The length is bumped by the CTA
+// of the sequence that takes the last of the atomic tickets every CTA takes
+// once it has read the old length (early in the kernel).
 //
 // Launch latency: the split geometry comes from the host (it mirrors the
 // lengths), so length, page table and the first copies are in flight together.
