@@ -221,7 +221,7 @@ void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float
                    int32_t *kept_count, int seg_base, int fill_pages, float *prio, const float *noise, int noise_stride,
                    int noise_base, cudaStream_t st) {
   // Variant by the longest segment: registers hold a whole segment up to 2048 (256-thread CTAs, many per SM), 8192
-  // (two CTAs per SM) or 32768 keys; longer segments stream their rounds from L2.
+  // (two CTAs per SM) or 32768 keys, a pair of CTAs 65536; longer segments stream their rounds from L2.
 #define FKV_SEL(S, M, T, P) \
   k_select<S, M, T, P><<<nblocks, T, 0, st>>>(c->ctx, scores, idx, kept_count, seg_base, fill_pages, prio, noise, \
                                              noise_stride, noise_base)
@@ -231,6 +231,23 @@ void launch_select(fkv_cache *c, int mode, int max_old, int nblocks, const float
     if (mode == 0) FKV_SEL(true, 0, kSelSmallThreads, kSelSmallPerThread); else FKV_SEL(true, 1, kSelSmallThreads, kSelSmallPerThread);
   } else if (max_old <= kSelRound) {
     if (mode == 0) FKV_SEL(true, 0, kSelThreads, 32); else FKV_SEL(true, 1, kSelThreads, 32);
+  } else if (max_old <= 2 * kSelRound) {
+    // Up to 65536 keys: a pair of CTAs (one cluster) per segment, each with half of the keys in registers.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * nblocks);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (mode == 0)
+      (void)cudaLaunchKernelEx(&cfg, k_select<true, 0, kSelThreads, 32, true>, c->ctx, scores, idx, kept_count, seg_base,
+                               fill_pages, prio, noise, noise_stride, noise_base);
+    else
+      (void)cudaLaunchKernelEx(&cfg, k_select<true, 1, kSelThreads, 32, true>, c->ctx, scores, idx, kept_count, seg_base,
+                               fill_pages, prio, noise, noise_stride, noise_base);
   } else {
     if (mode == 0) FKV_SEL(false, 0, kSelThreads, 32); else FKV_SEL(false, 1, kSelThreads, 32);
   }

@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(1024) k_golden_select(const float *alpha, int 
     uint32_t Tk;
     unsigned need;
     int nv = nm;
-    sel_kth_key<1024, kPer>(sh, key, nv, 1, [](int) {}, (unsigned)k, Tk, need);
+    sel_kth_key<1024, kPer>(sh, key, nv, 1, [](int) {}, SelAlone{}, (unsigned)k, Tk, need);
     unsigned long long total;
     const unsigned long long excl = sel_counts_before<1024, kPer>(sh, key, nv, Tk, total);   // its barriers: every thread has read its cache entries
     unsigned bgt = (unsigned)(excl & 0xffffffffu), beq = (unsigned)(excl >> 32);

@@ -4,7 +4,7 @@
 // are written in ascending order, which is the order compaction needs.
 //
 // Integer work on 4 bytes per pair, read from L2 right after the scorer wrote
-// them.  One CTA per segment: a histogram select finds the k-th largest key T
+// them.  One CTA per segment (a cluster of two for 32769 .. 65536 competing pairs): a histogram select finds the k-th largest key T
 // and how many pairs equal to T are still needed; one ordered pass then emits
 // {key > T} plus the first `need` slots with key == T, using block prefix
 // sums - no atomics decide which tied pair stays.
@@ -77,6 +77,33 @@ struct SelShared {
   unsigned red[64];
   unsigned bin, krem;
   unsigned long long wsum[33];
+  unsigned long long xch[2];   // what a CTA pair tells each other: (min, max) of the keys; the first CTA's totals
+};
+
+// How the CTAs that share one segment's selection combine what each of them knows.  One CTA on its own: nothing to do.
+struct SelAlone {
+  template <int THREADS> __device__ __forceinline__ void minmax(SelShared<THREADS> &, uint32_t &, uint32_t &) const {}
+  __device__ __forceinline__ void hist_ready() const {}
+  template <int THREADS> __device__ __forceinline__ unsigned bin(const SelShared<THREADS> &sh, int b) const { return sh.hist[b]; }
+  __device__ __forceinline__ void hist_read() const {}
+};
+// Two CTAs of one cluster, each with half of the segment's keys in registers: both see both halves' minimum and
+// maximum and the sum of both histograms (read from the other CTA's shared memory), and so take the same decisions.
+// Every thread of both CTAs makes every call (cluster barriers inside).
+struct SelPair {
+  uint32_t peer;   // the other CTA's rank in the cluster
+  template <int THREADS> __device__ __forceinline__ void minmax(SelShared<THREADS> &sh, uint32_t &kmin, uint32_t &kmax) const {
+    if (threadIdx.x == 0) sh.xch[0] = (unsigned long long)kmin | ((unsigned long long)kmax << 32);
+    cluster_sync_all();
+    const unsigned long long o = dsmem_ld_u64(dsmem_addr(smem_u32(&sh.xch[0]), peer));
+    kmin = min(kmin, (uint32_t)(o & 0xffffffffu));
+    kmax = max(kmax, (uint32_t)(o >> 32));
+  }
+  __device__ __forceinline__ void hist_ready() const { cluster_sync_all(); }   // both histograms are complete
+  template <int THREADS> __device__ __forceinline__ unsigned bin(const SelShared<THREADS> &sh, int b) const {
+    return sh.hist[b] + dsmem_ld_u32(dsmem_addr(smem_u32(&sh.hist[b]), peer));
+  }
+  __device__ __forceinline__ void hist_read() const { cluster_sync_all(); }    // ... and may be cleared again
 };
 
 // The k-th largest key T of the keys the CTA holds (0 < k < their number) and how many keys EQUAL to T
@@ -86,9 +113,9 @@ struct SelShared {
 // 2 x THREADS equal bins (the bins follow the data, not fixed bit fields, so shared-memory atomics
 // spread out), picks the bin where the count from the top crosses k and narrows the window to it -
 // at most three passes for 32-bit keys.
-template <int THREADS, int PER, class Reload>
+template <int THREADS, int PER, class Reload, class Exch>
 __device__ __forceinline__ void sel_kth_key(SelShared<THREADS> &sh, uint32_t (&key)[PER], int &nv, int rounds,
-                                            Reload reload, unsigned k, uint32_t &T, unsigned &need) {
+                                            Reload reload, const Exch &exch, unsigned k, uint32_t &T, unsigned &need) {
   constexpr int kBins = 2 * THREADS, NWARPS = THREADS / 32;
   constexpr int kLogBins = THREADS == 1024 ? 11 : THREADS == 512 ? 10 : 9;
   static_assert(THREADS == 1024 || THREADS == 512 || THREADS == 256, "bins = 2 x threads, a power of two");
@@ -106,6 +133,7 @@ __device__ __forceinline__ void sel_kth_key(SelShared<THREADS> &sh, uint32_t (&k
   __syncthreads();
   kmin = __reduce_min_sync(0xffffffffu, lane < NWARPS ? sh.red[lane] : 0xffffffffu);
   kmax = __reduce_max_sync(0xffffffffu, lane < NWARPS ? sh.red[32 + lane] : 0u);
+  exch.minmax(sh, kmin, kmax);
   T = kmin;
   need = k;
   if (kmin == kmax) return;
@@ -125,9 +153,10 @@ __device__ __forceinline__ void sel_kth_key(SelShared<THREADS> &sh, uint32_t (&k
       }
     }
     __syncthreads();
+    exch.hist_ready();
     // Bins in descending order, two per thread: the top one is 2 THREADS - 1 - 2 tid.
     {
-      const unsigned v0 = sh.hist[kBins - 1 - 2 * tid], v1 = sh.hist[kBins - 2 - 2 * tid];
+      const unsigned v0 = exch.bin(sh, kBins - 1 - 2 * tid), v1 = exch.bin(sh, kBins - 2 - 2 * tid);
       int tot;
       const unsigned above = (unsigned)block_excl_scan((int)(v0 + v1), sh.scan, tot);
       if (above < krem && krem <= above + v0) {
@@ -137,6 +166,7 @@ __device__ __forceinline__ void sel_kth_key(SelShared<THREADS> &sh, uint32_t (&k
       }
     }
     __syncthreads();
+    exch.hist_read();
     lo += sh.bin << shift;
     krem = sh.krem;
     __syncthreads();
@@ -194,39 +224,49 @@ __device__ __forceinline__ int sel_place(bool greater, bool equal, unsigned bgt,
   return -1;
 }
 
-template <bool SINGLE, int MODE, int THREADS, int PER>
+// PAIR: two CTAs (one cluster, consecutive block indices) share a segment of up to 2 x THREADS x PER competing pairs:
+// each holds one half of the keys in registers for every pass, the histograms are summed across the pair through
+// distributed shared memory, and the second CTA's places start after the first one's counts.
+template <bool SINGLE, int MODE, int THREADS, int PER, bool PAIR = false>
 __global__ void __launch_bounds__(THREADS) k_select(Ctx c, const float *scores, int32_t *idx, int32_t *kept_count,
                                                          int seg_base, int fill_pages, float *prio,
                                                          const float *noise, int noise_stride, int noise_base) {
   constexpr int kSelPerThread = PER, kSelRound = THREADS * PER;
   __shared__ SelShared<THREADS> sh;
-  if ((int)blockIdx.x >= c.planhdr[PH_NWORK]) return;
-  const int seg = c.work[blockIdx.x];
+  static_assert(!PAIR || SINGLE, "a CTA of a pair keeps its half in registers");
+  const int witem = PAIR ? blockIdx.x >> 1 : blockIdx.x, half = PAIR ? blockIdx.x & 1 : 0;
+  if (witem >= c.planhdr[PH_NWORK]) return;   // (both CTAs of a pair)
+  const int seg = c.work[witem];
   const SegPlan p = c.plan[seg];
   const int tid = threadIdx.x;
-  if (fill_pages) fill_pt_new(c, seg, p);
+  if (fill_pages && half == 0) fill_pt_new(c, seg, p);
   const int m = p.n_old - p.r;
   const int k = MODE == 0 ? p.k_sel : max(0, m - 2 * (p.n_old - p.n_new));   // MODE 1: the non-candidates
   const float *sc = scores + (size_t)(seg - seg_base) * c.cap;
   int32_t *out = MODE == 0 ? idx + (size_t)(seg - seg_base) * c.cap : nullptr;
   float *pr = MODE == 1 ? prio + (size_t)(seg - seg_base) * c.cap : nullptr;
   const float *nz = MODE == 1 ? noise + (size_t)(seg - noise_base) * noise_stride : nullptr;
+  // The cases that need no search (the first CTA of a pair writes them; both leave).
   if (MODE == 0) {
-    if (kept_count && tid == 0) kept_count[seg - seg_base] = p.n_new;
+    if (kept_count && tid == 0 && half == 0) kept_count[seg - seg_base] = p.n_new;
     // The protected recent slots close the list.
-    for (int j = tid; j < p.r; j += THREADS) out[k + j] = m + j;
+    if (half == 0)
+      for (int j = tid; j < p.r; j += THREADS) out[k + j] = m + j;
     if (k <= 0) return;
     if (k >= m) {
-      for (int j = tid; j < m; j += THREADS) out[j] = j;
+      if (half == 0)
+        for (int j = tid; j < m; j += THREADS) out[j] = j;
       return;
     }
   } else {
     if (k <= 0) {   // every competing pair is a candidate: rank = slot
-      for (int j = tid; j < m; j += THREADS) pr[j] = key_score(score_key(sc[j])) - nz[j];
+      if (half == 0)
+        for (int j = tid; j < m; j += THREADS) pr[j] = key_score(score_key(sc[j])) - nz[j];
       return;
     }
     if (k >= m) {   // nothing to evict
-      for (int j = tid; j < m; j += THREADS) pr[j] = INFINITY;
+      if (half == 0)
+        for (int j = tid; j < m; j += THREADS) pr[j] = INFINITY;
       return;
     }
   }
@@ -246,11 +286,12 @@ __global__ void __launch_bounds__(THREADS) k_select(Ctx c, const float *scores, 
       key[4 * q + 2] = score_key(x[q].z); key[4 * q + 3] = score_key(x[q].w);
     }
   };
-  if (SINGLE) load_round(0);
+  if (SINGLE) load_round(half);   // (a CTA of a pair: its half of the keys)
 
   uint32_t T;
   unsigned need;
-  sel_kth_key<THREADS, PER>(sh, key, nv, rounds, load_round, (unsigned)k, T, need);
+  if (PAIR) sel_kth_key<THREADS, PER>(sh, key, nv, rounds, load_round, SelPair{(uint32_t)(half ^ 1)}, (unsigned)k, T, need);
+  else sel_kth_key<THREADS, PER>(sh, key, nv, rounds, load_round, SelAlone{}, (unsigned)k, T, need);
 
   // ---- ordered emit: one block prefix sum per round ----
   unsigned run_gt = 0, run_eq = 0;
@@ -258,8 +299,17 @@ __global__ void __launch_bounds__(THREADS) k_select(Ctx c, const float *scores, 
     if (!SINGLE) load_round(round);
     unsigned long long tot;
     const unsigned long long excl = sel_counts_before<THREADS, PER>(sh, key, nv, T, tot);
+    if (PAIR) {   // the second CTA's places start after the first one's counts
+      if (half == 0 && tid == 0) sh.xch[1] = tot;
+      cluster_sync_all();
+      if (half == 1) {
+        const unsigned long long first = dsmem_ld_u64(dsmem_addr(smem_u32(&sh.xch[1]), 0));
+        run_gt = (unsigned)(first & 0xffffffffu); run_eq = (unsigned)(first >> 32);
+      }
+      cluster_sync_all();   // the first CTA's shared memory has been read: it may leave
+    }
     unsigned bgt = run_gt + (unsigned)(excl & 0xffffffffu), beq = run_eq + (unsigned)(excl >> 32);
-    const int slot0 = round * kSelRound + tid * kSelPerThread;
+    const int slot0 = (PAIR ? half : round) * kSelRound + tid * kSelPerThread;
 #pragma unroll
     for (int j = 0; j < kSelPerThread; ++j) {
       const bool g = j < nv && key[j] > T, e = j < nv && key[j] == T;
