@@ -295,9 +295,11 @@ def test_config5_layer_slice():
 
 
 @pytest.mark.parametrize("n,B,R", [(40000, 10000, 0), (65536, 16384, 0), (70001, 3, 5), (32769, 32768, 0),
-                                   (65536, 16384, 256)])
+                                   (65536, 16384, 256), (65536, 1, 0), (50000, 49000, 0), (33000, 32999, 7),
+                                   (65536, 65535, 0), (65537, 30000, 1), (131072, 5000, 0)])
 def test_select_long_segments_bit_exact(n, B, R):
-    # Segments longer than one selection round (32768 keys): the multi-round path.
+    # Segments longer than one CTA's registers hold (32768 keys): a pair of CTAs up to 65536 competing pairs (both
+    # sides of its limits, one key to keep, one key to drop), rounds streamed from L2 beyond.
     w = wl.Workload("sel_long", 1, 2, 4, 64, (n,), (B,), R, 12, "normal")
     c = binding.from_workload(w)
     K, V, A, pos = wl.layer_inputs(w, 0, 0, "cuda")

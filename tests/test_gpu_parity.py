@@ -600,7 +600,8 @@ def test_fused_append_without_free_pages_moves_no_head(free_pages):
 
 # ------------------------------------------------------------------ the sampled action (Section 3.1, Eq. 2; App. B.2)
 @pytest.mark.parametrize("n,B,R", [(512, 256, 0), (600, 344, 32), (5000, 4744, 0), (4097, 4096, 0), (9000, 8744, 256),
-                                   (300, 300, 0), (777, 100, 100), (1000, 600, 0), (40000, 39000, 0), (70001, 60000, 5)])
+                                   (300, 300, 0), (777, 100, 100), (1000, 600, 0), (40000, 39000, 0), (70001, 60000, 5),
+                                   (65536, 49152, 0), (65536, 65000, 256)])
 @pytest.mark.parametrize("fn", [_normal, _ties, _special])
 def test_select_sampled_bit_exact(n, B, R, fn):
     # Given the same scores and the same Gumbel draws the kept list is the oracle's, bit for bit
