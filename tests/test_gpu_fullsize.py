@@ -110,7 +110,7 @@ def all_layers_properties(ld):
                     assert p[-r:].tolist() == list(range(w.lens[s] - r, w.lens[s]))
 
 
-def check_every_segment(ld, gpu_scores):
+def check_every_segment(ld, gpu_scores, layers=None):
     """After an all-layer eviction: every (layer, sequence, KV head) against the oracle, then one decode
     token over every segment.  The inputs of a layer are generated again from their seeds (the same
     bytes the cache was filled with) and the oracle's whole eviction step runs over the layer's
@@ -121,7 +121,7 @@ def check_every_segment(ld, gpu_scores):
     w, g = ld.w, ld.w.group_size
     Hk, R = w.num_kv_heads, w.recent_keep
     compared, worst_score, worst_attn = 0, 0.0, 0.0
-    for l in range(ld.L):
+    for l in range(layers or ld.L):
         W1, b1, W2, b2 = (npf(t) for t in wl.scorer_params(w, l, "cuda"))
         Ks, Vs, As, ps, ns, Bs, w1s, b1s, w2s, b2s, where = [], [], [], [], [], [], [], [], [], [], []
         for s in range(w.batch):
@@ -285,12 +285,14 @@ def test_config5_layer_slice():
         u = sc[:w.lens[s]].view(np.uint32)
         for gidx in np.where(cnt > 1)[0][:200]:
             assert len(set(u[inv == gidx].tolist())) == 1
+    full = {l: npf(ld.cache.score(l)) for l in range(2)}   # every segment of the first two layers, sampled ones of the rest
     ld.cache.evict(binding.ALL_LAYERS)
     for l, s, h in samples:
         check_evicted_segment(ld, l, s, h, gs[(l, s, h)])
     all_layers_properties(ld)
     for l, s, h in samples:
         check_attention(ld, l, [(s, h)])
+    assert check_every_segment(ld, full, layers=2) == 2 * w.batch * w.num_kv_heads    # 128 segments of 65536 pairs
     assert ld.cache.device_status()[0] == 0
 
 
