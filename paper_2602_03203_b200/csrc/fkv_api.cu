@@ -151,6 +151,8 @@ struct fkv_cache {
   int max_cluster = 0;        // largest attention cluster the device places (found at the first stand-alone launch)
   float feature_scale = 0.f;  // softmax scale of the recorded queries (the last decode call's)
   bool timing = false, timed = false;
+  CUtensorMap k_rows;         // the page pool's K rows as [page][row][64-channel half][64 channels] (R-KV's tensor copies)
+  bool k_rows_ready = false;
   cudaEvent_t ev[7] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};  // [6]: after the plan
 };
 
@@ -282,6 +284,36 @@ int launch_features(fkv_cache *c, int max_old, int nwork_bound, cudaStream_t st)
                                 : launch_features_t<64>(c, max_old, nwork_bound, scale_log2, st);
 }
 
+// The tensor map of R-KV's copies: bf16 [num_pages][16 rows][D / 64 halves][64 channels] over the page pool, one box =
+// the 16 rows x 64 channels of one page (2 KB, 16 rows of 128 bytes in shared memory; the record's own chunk swizzle
+// stays as it is).  The driver's encoder is reached through the runtime, so the library links no driver stub.
+int ensure_k_rows_map(fkv_cache *c) {
+  if (c->k_rows_ready) return FKV_OK;
+  typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult found;
+  FKV_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &found));
+  if (fn == nullptr || found != cudaDriverEntryPointSuccess) {
+    g_cuda_error = "cuTensorMapEncodeTiled is not available from this driver";
+    return FKV_ERR_CUDA;
+  }
+  const int D = c->cfg.head_dim;
+  const cuuint64_t dims[4] = {64, (cuuint64_t)(D / 64), (cuuint64_t)kPage, (cuuint64_t)c->ctx.num_pages};
+  const cuuint64_t strides[3] = {128, (cuuint64_t)(4 * D), (cuuint64_t)c->ctx.page_bytes};   // bytes, dimensions 1 .. 3
+  const cuuint32_t box[4] = {64, 1, (cuuint32_t)kPage, 1}, step[4] = {1, 1, 1, 1};
+  const CUresult r = reinterpret_cast<encode_fn>(fn)(&c->k_rows, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, c->ctx.pool, dims, strides,
+                                                     box, step, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_cuda_error = "cuTensorMapEncodeTiled failed with driver error " + std::to_string((int)r);
+    return FKV_ERR_CUDA;
+  }
+  c->k_rows_ready = true;
+  return FKV_OK;
+}
+
 // R-KV baseline scores of the segments on the work list (after a k_plan): the attention term and the reciprocal
 // key norms first (the index scratch holds the norms until the selection overwrites it), then the n x n
 // contraction.  Work items sit on grid.x (no 65535 limit).
@@ -289,6 +321,7 @@ template <int D>
 int launch_rkv_t(fkv_cache *c, float *out, int seg_base, int max_old, int nwork_bound, long long tiles, float la, float ls,
                  cudaStream_t st) {
   if (max_old <= 0 || nwork_bound <= 0) return FKV_OK;
+  if (int e = ensure_k_rows_map(c)) return e;
   float *rn = reinterpret_cast<float *>(c->ctx.idx);
   k_rkv_prepare<D><<<dim3(nwork_bound, (max_old + 127) / 128), 128, 0, st>>>(c->ctx, out, rn, seg_base,
                                                                              FKV_FEATURE_WINDOW8);
@@ -297,7 +330,7 @@ int launch_rkv_t(fkv_cache *c, float *out, int seg_base, int max_old, int nwork_
   static SmemOptIn opt_in;
   FKV_CUDA(opt_in.ensure(k_rkv_score<D>, smem));
   const int grid = (int)std::max<long long>(1, std::min<long long>(c->sm_count, tiles));
-  k_rkv_score<D><<<grid, kRkvThreads, smem, st>>>(c->ctx, out, rn, seg_base, la, ls);
+  k_rkv_score<D><<<grid, kRkvThreads, smem, st>>>(c->ctx, c->k_rows, out, rn, seg_base, la, ls);
   FKV_LAUNCHED(c);
   return FKV_OK;
 }

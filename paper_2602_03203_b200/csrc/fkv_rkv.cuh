@@ -10,37 +10,51 @@
 // contraction, 2 n^2 D flops per segment (275 GFLOP at n = 32768, D = 128) against 2 n D bytes of keys that stay
 // in L2 - compute-bound, so it runs on the 5th-generation tensor cores.  Nothing of the n x n matrix is ever
 // stored: a CTA holds 256 rows (two M = 128 operand tiles) in shared memory, streams the segment's keys past
-// them 128 at a time, and reduces every 128 x 128 block of products in the epilogue that reads it from tensor
+// them 256 at a time, and reduces every 128 x 256 block of products in the epilogue that reads it from tensor
 // memory.
 //
 // One persistent CTA per SM over a contiguous range of the plan's 128-pair tiles, taken two at a time:
-//   warps 0-3   copy K rows of page records into K-major operand tiles (16-byte asynchronous copies; the page
-//               record's swizzle is the shared-memory swizzle), the CTA's 256 rows once, then the column tiles
-//               into a ring, with the column tile's reciprocal norms;
-//   warp 4      one lane issues tcgen05.mma (bf16 x bf16 -> fp32, M = N = 128, K = 16 per instruction) into one of
-//               two pairs of accumulators in tensor memory and hands them on with tcgen05.commit;
-//   warps 8-15  two warpgroups, one per 128 rows: a thread owns one row (its tensor-memory lane), scales the
-//               products by the column's reciprocal norm and keeps the running maximum; the diagonal and the
-//               columns past the segment's end are masked in the two tiles that have them.
+//   warp 0      tensor copies (TMA) of K rows out of page records: one copy = the 16 rows x 64 channels of one page
+//               (the tensor map sees the page pool as [page][row][64-channel half][64 channels]), 2 KB that land as
+//               16 rows of a K-major operand tile - the page record's swizzle is the shared-memory swizzle.  A lane
+//               per copy: the unit's 256 rows once, then the column tiles into a ring, with their reciprocal norms;
+//   warp 1      one lane issues tcgen05.mma (bf16 x bf16 -> fp32, M = 128, N = 256, K = 16 per instruction: an
+//               instruction takes about 130 cycles whatever its N up to 128, and 155 at N = 256) into one of the
+//               two 256-column accumulators of tensor memory and hands them on with tcgen05.commit;
+//   warps 4-11  reduce: warp = 32 rows (its tensor-memory lanes) x 128 of the 256 columns; a thread scales the
+//               products by the column's reciprocal norm and keeps the running maximum of its row, the next 32
+//               columns on their way from tensor memory meanwhile; the diagonal and the columns past the segment's
+//               end are masked in the tiles that have them.  The two column halves of a row meet at the unit's end.
 // Reciprocal norms and the attention term come from a small kernel that runs before (one thread per pair).
 // Every wait is bounded; tensor memory is freed at the common exit.
 #pragma once
+#include <cuda.h>
 #include "fkv_dev.cuh"
 #include "fkv_features.cuh"
 
 namespace fkv {
 
-constexpr int kRkvStages = 4;                 // column tiles in flight
-constexpr int kRkvNormSlots = kRkvStages + 3; // the copies run at most kRkvStages ahead of the mma, the mma at most 2 ahead of the reduction
-constexpr int kRkvThreads = 16 * 32;
+constexpr int kRkvStages = 2;                 // column tiles (256 keys) in the ring
+constexpr int kRkvCols = 256;                 // keys per column tile = N of the mma
+constexpr int kRkvNormSlots = kRkvStages + 2; // the copies run at most kRkvStages ahead of the mma, the mma at most one tile ahead of the reduction
+constexpr int kRkvXch = 4;                    // hand-over slots of the row maxima (by unit)
+constexpr int kRkvThreads = 12 * 32;
 
 struct RkvSmem {
-  static __host__ __device__ size_t tile(int D) { return (size_t)(D / 64) * 128 * 128; }   // [D/64][128 rows][128 B]
-  // 1 KB alignment slack | A (two tiles) | B ring | reciprocal norms | barriers
+  static __host__ __device__ size_t tile(int D) { return (size_t)(D / 64) * 128 * 128; }   // 128 rows: [D/64][128][128 B]
+  // 1 KB alignment slack | A (two tiles) | B ring (two tiles' worth a stage) | reciprocal norms | row maxima | barriers
   static __host__ __device__ size_t bytes(int D) {
-    return 1024 + (2 + kRkvStages) * tile(D) + (size_t)kRkvNormSlots * 128 * 4 + 256;
+    return 1024 + (2 + 2 * kRkvStages) * tile(D) + (size_t)kRkvNormSlots * kRkvCols * 4 + (size_t)kRkvXch * 256 * 4 + 256;
   }
 };
+
+// One page's K rows, channels 64 q .. 64 q + 63, to 16 consecutive 128-byte rows of an operand tile.
+__device__ __forceinline__ void tma_page_k(uint32_t dst, const CUtensorMap *tm, int q, int page, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(0), "r"(q), "r"(0), "r"(page), "r"(bar)
+      : "memory");
+}
 
 // Before the contraction: thread = pair.  rn[seg * cap + slot] = 1 / |k| (0 for a zero key), and the attention term
 // (feature `column` averaged over the g heads, summed in head order and divided in fp32) into
@@ -78,7 +92,7 @@ struct RkvWalk {
   int wi, tbeg, tend, seg, n;
 };
 struct RkvUnit {
-  int row0, halves, ntj;   // first row, 128-row halves in use (1 or 2), column tiles of the segment
+  int row0, halves, ntj;   // first row, 128-row halves in use (1 or 2), 256-key column tiles of the segment
 };
 __device__ __forceinline__ int rkv_unit(const Ctx &c, int t, int t1, RkvWalk &w, RkvUnit &u) {   // returns tiles taken
   if (t >= w.tend) {
@@ -89,14 +103,16 @@ __device__ __forceinline__ int rkv_unit(const Ctx &c, int t, int t1, RkvWalk &w,
   }
   u.row0 = (t - w.tbeg) * 128;
   u.halves = (t + 1 < w.tend && t + 1 < t1) ? 2 : 1;
-  u.ntj = (w.n + 127) / 128;
+  u.ntj = (w.n + kRkvCols - 1) / kRkvCols;
   return u.halves;
 }
 
+
 template <int D>
-__global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, float *out, const float *rn, int seg_base,
-                                                              float lambda_a, float lambda_s) {
-  constexpr int NCH = D / 8, RSTEP = 128 / NCH, NST = kRkvStages, NR = kRkvNormSlots;
+__global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __grid_constant__ CUtensorMap tmk, float *out,
+                                                              const float *rn, int seg_base, float lambda_a, float lambda_s) {
+  constexpr int NQ = D / 64, NST = kRkvStages, NR = kRkvNormSlots, NC = kRkvCols;
+  constexpr uint32_t PAGE_HALF = kPage * 128;   // bytes of one tensor copy
   extern __shared__ uint8_t smem_raw[];
   const int total = c.planhdr[PH_TILES1], nwork = c.planhdr[PH_NWORK];
   const int per = (total + (int)gridDim.x - 1) / (int)gridDim.x;
@@ -106,19 +122,21 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, float *out,
 
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const size_t tb = RkvSmem::tile(D);
-  uint8_t *At = smem;                                    // [2][HALVES][128][128 B]
-  uint8_t *Bt = At + 2 * tb;                             // [NST][HALVES][128][128 B]
-  float *Rn = reinterpret_cast<float *>(Bt + NST * tb);  // [NR][128]
-  uint64_t *bars = reinterpret_cast<uint64_t *>(Rn + NR * 128);
+  uint8_t *At = smem;                                        // [2][D/64][128 rows][128 B]
+  uint8_t *Bt = At + 2 * tb;                                 // [NST][D/64][256 rows][128 B]
+  float *Rn = reinterpret_cast<float *>(Bt + NST * 2 * tb);  // [NR][256]
+  float *Xch = Rn + NR * NC;                                 // [kRkvXch][2 halves][128 rows]
+  uint64_t *bars = reinterpret_cast<uint64_t *>(Xch + kRkvXch * 256);
   uint64_t *a_full = bars, *a_empty = bars + 1, *b_full = bars + 2, *b_empty = b_full + NST;
-  uint64_t *acc_full = b_empty + NST, *acc_empty = acc_full + 2;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+  uint64_t *acc_full = b_empty + NST, *acc_empty = acc_full + 2, *x_full = acc_empty + 2;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(x_full + kRkvXch);
 
-  if (warp == 0) tmem_alloc(smem_u32(tmem_slot), 512);   // two pairs of 128-column accumulators
+  if (warp == 0) tmem_alloc(smem_u32(tmem_slot), 512);   // two accumulators of 256 columns
   if (threadIdx.x == 0) {
-    mbar_init(smem_u32(a_full), 128); mbar_init(smem_u32(a_empty), 1);
-    for (int s = 0; s < NST; ++s) { mbar_init(smem_u32(&b_full[s]), 128); mbar_init(smem_u32(&b_empty[s]), 1); }
+    mbar_init(smem_u32(a_full), 1); mbar_init(smem_u32(a_empty), 1);
+    for (int s = 0; s < NST; ++s) { mbar_init(smem_u32(&b_full[s]), 1); mbar_init(smem_u32(&b_empty[s]), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&acc_full[b]), 1); mbar_init(smem_u32(&acc_empty[b]), 8); }
+    for (int x = 0; x < kRkvXch; ++x) mbar_init(smem_u32(&x_full[x]), 4);
     fence_barrier_init();
   }
   tc_fence_before();
@@ -131,153 +149,181 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, float *out,
   w.tend = -1;
   RkvUnit u;
 
-  if (warp < 4) {
-    // ---------------- copies: thread = one 16-byte chunk column of rows R0, R0 + RSTEP, ... of every page ----------------
-    const int p = threadIdx.x, ch = p % NCH, R0 = p / NCH;
-    const uint32_t dcol = (uint32_t)((ch >> 3) * 128 * 128 + (ch & 7) * 16);
-    // One 128-row tile of the segment (its pages pg0 ..) into the operand tile at dst.
-    auto copy_tile = [&](uint32_t dst, int pg0) {
-      const int np = min(8, (w.n + kPage - 1) / kPage - pg0);
-      const int *ptrow = c.pt + (size_t)w.seg * c.max_pages + pg0;
-      int pid[8];
-#pragma unroll
-      for (int pg = 0; pg < 8; ++pg) pid[pg] = ptrow[min(pg, max(np - 1, 0))];
-#pragma unroll
-      for (int pg = 0; pg < 8; ++pg) {
-        if (pg < np) {
-          const uint8_t *page = c.pool + (size_t)pid[pg] * c.page_bytes + ch * 16;
-#pragma unroll
-          for (int k = 0; k < kPage / RSTEP; ++k) {
-            const int r = R0 + k * RSTEP;
-            cp_async16(dst + dcol + (uint32_t)((pg * kPage + r) * 128), page + r * 4 * D);
-          }
-        }
-      }
-    };
-    // The column tiles are copied two ahead: the copies of tile j are issued before those of tile j - 2 are waited
-    // for (a copy from L2 takes longer than the multiplies of a tile), and a tile is handed over - this thread's
-    // copies complete, made visible to the tensor core's reads, one arrival - two tiles after it was asked for.
-    FeatRing br{0, 0}, done{0, 0};
+  if (warp == 0) {
+    // ---------------- copies: a lane per tensor copy (one page x one 64-channel half) ----------------
+    FeatRing br{0, 0};
     int nu = 0, jr = 0;   // units so far (phase of the A barriers); ring slot of the next column tile's norms
+    int armed_a = -1;                       // parity of the last phase armed on the barrier of the unit's rows
+    uint32_t armed_b = 0, armed_par = 0;    // ... and of the column tiles' stages: bit s = stage s armed at all / its parity
     bool ok = true;
-    auto hand_over = [&]() {
-      fence_proxy_async();
-      mbar_arrive(smem_u32(&b_full[done.i]));
-      done.next(NST);
-    };
     for (int t = t0; t < t1 && ok;) {
       const int took = rkv_unit(c, t, t1, w, u);
-      if (!mbar_wait_warp(smem_u32(a_empty), (nu & 1) ^ 1)) { set_status(c, kDevWaitTimeout); break; }
-      for (int h = 0; h < u.halves; ++h) copy_tile(smem_u32(At + h * tb), (u.row0 + h * 128) / kPage);
-      cp_async_wait_all();
-      fence_proxy_async();
-      mbar_arrive(smem_u32(a_full));
-      int inflight = 0;
+      const int npg = (w.n + kPage - 1) / kPage;
+      const int *ptrow = c.pt + (size_t)w.seg * c.max_pages;
+      {
+        // The unit's rows: lane = (half of the unit, page of the half, channel half).
+        const int h = lane >> 4, pg = (lane >> 1) & 7, q = lane & 1;
+        const int pa = u.row0 / kPage + h * 8 + pg;
+        const bool on = h < u.halves && pa < npg && q < NQ;
+        const int pid = on ? ptrow[pa] : 0;
+        const int ncopies = __popc(__ballot_sync(0xffffffffu, on));
+        if (!mbar_wait_warp(smem_u32(a_empty), (nu & 1) ^ 1)) { set_status(c, kDevWaitTimeout); break; }
+        if (lane == 0) mbar_arrive_expect_tx(smem_u32(a_full), (uint32_t)ncopies * PAGE_HALF);
+        armed_a = nu & 1;
+        __syncwarp();
+        if (on) tma_page_k(smem_u32(At + h * tb + (size_t)q * 128 * 128 + (size_t)pg * PAGE_HALF), &tmk, q, pid, smem_u32(a_full));
+      }
+      // Column tiles: lane = (channel half, page of the tile); the page id is read one tile before its copy.
+      const int pg = lane & 15, q = lane >> 4;
+      int pidn = (pg < npg && q < NQ) ? ptrow[pg] : 0;
       for (int j = 0; j < u.ntj; ++j) {
+        const int pb = j * 16 + pg;
+        const bool on = pb < npg && q < NQ;
+        const int pid = pidn;
+        if (j + 1 < u.ntj) pidn = (pb + 16 < npg && q < NQ) ? ptrow[pb + 16] : 0;
+        const int ncopies = __popc(__ballot_sync(0xffffffffu, on));
         if (!mbar_wait_warp(smem_u32(&b_empty[br.i]), br.ph ^ 1)) { set_status(c, kDevWaitTimeout); ok = false; break; }
-        copy_tile(smem_u32(Bt + br.i * tb), j * 8);
-        if (p < 32 && j * 128 + p * 4 < c.cap)   // this tile's reciprocal norms (entries past the segment's end are masked later)
-          cp_async16(smem_u32(Rn + jr * 128 + p * 4), rn + (size_t)w.seg * c.cap + j * 128 + p * 4);
-        cp_async_commit();
+        const uint32_t nbytes = (uint32_t)min(NC, c.cap - j * NC) * 4u;   // reciprocal norms (entries past the segment's end are masked later)
+        if (lane == 0) mbar_arrive_expect_tx(smem_u32(&b_full[br.i]), (uint32_t)ncopies * PAGE_HALF + nbytes);
+        armed_b |= 1u << br.i;
+        armed_par = (armed_par & ~(1u << br.i)) | ((uint32_t)br.ph << br.i);
+        __syncwarp();
+        if (on) tma_page_k(smem_u32(Bt + (size_t)br.i * 2 * tb + (size_t)q * NC * 128 + (size_t)pg * PAGE_HALF), &tmk, q, pid, smem_u32(&b_full[br.i]));
+        if (lane == 0) bulk_g2s(smem_u32(Rn + jr * NC), rn + (size_t)w.seg * c.cap + (size_t)j * NC, nbytes, smem_u32(&b_full[br.i]));
         br.next(NST);
         if (++jr == NR) jr = 0;
-        if (++inflight == 3) {
-          cp_async_wait_pending<2>();
-          hand_over();
-          --inflight;
-        }
       }
-      // The last tiles of the unit (on a failed wait too: nothing may be in flight at the exit).
-      cp_async_wait_pending<0>();
-      for (; inflight > 0 && ok; --inflight) hand_over();
       ++nu;
       t += took;
     }
-  } else if (warp == 4 && lane == 0) {
-    // ---------------- multiplies ----------------
-    const uint32_t idesc = umma_idesc_bf16(128, 128);
+    // No copy may be in flight at the exit: every armed phase has completed (at once on the ordinary way out, where
+    // the multiplies have waited for each of them).
+    if (armed_a >= 0 && !mbar_wait_warp(smem_u32(a_full), (uint32_t)armed_a)) set_status(c, kDevWaitTimeout);
+#pragma unroll
+    for (int s = 0; s < NST; ++s)
+      if (((armed_b >> s) & 1u) && !mbar_wait_warp(smem_u32(&b_full[s]), (armed_par >> s) & 1u)) set_status(c, kDevWaitTimeout);
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- multiplies: one item = (column tile, half) = one accumulator ----------------
+    const uint32_t idesc = umma_idesc_bf16(128, NC);
     FeatRing br{0, 0};
-    int nu = 0, uacc = 0;
+    int nu = 0, item = 0;
     bool ok = true;
     for (int t = t0; t < t1 && ok;) {
       const int took = rkv_unit(c, t, t1, w, u);
       if (!mbar_spin(smem_u32(a_full), nu & 1)) { set_status(c, kDevWaitTimeout); break; }
-      for (int j = 0; j < u.ntj; ++j, ++uacc) {
-        const int b = uacc & 1;
-        if (!mbar_spin(smem_u32(&b_full[br.i]), br.ph) || !mbar_spin(smem_u32(&acc_empty[b]), ((uacc >> 1) & 1) ^ 1)) {
-          set_status(c, kDevWaitTimeout); ok = false; break;
-        }
-        tc_fence_after();
-        const uint64_t bd0 = umma_desc_sw128(smem_u32(Bt + br.i * tb));
-        for (int h = 0; h < u.halves; ++h) {
+      for (int j = 0; j < u.ntj && ok; ++j) {
+        if (!mbar_spin(smem_u32(&b_full[br.i]), br.ph)) { set_status(c, kDevWaitTimeout); ok = false; break; }
+        const uint64_t bd0 = umma_desc_sw128(smem_u32(Bt + (size_t)br.i * 2 * tb));
+        for (int h = 0; h < u.halves; ++h, ++item) {
+          const int slot = item & 1;
+          if (!mbar_spin(smem_u32(&acc_empty[slot]), ((item >> 1) & 1) ^ 1)) { set_status(c, kDevWaitTimeout); ok = false; break; }
+          tc_fence_after();
           const uint64_t ad0 = umma_desc_sw128(smem_u32(At + h * tb));
-          const uint32_t d = tmem_base + (uint32_t)(b * 2 + h) * 128;
+          const uint32_t d = tmem_base + (uint32_t)slot * NC;
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {        // K = 16 channels per instruction: 32 bytes inside the swizzled row
-            const uint64_t off = (uint64_t)(((ks >> 2) * 128 * 128 + (ks & 3) * 32) >> 4);
-            umma_bf16(d, ad0 + off, bd0 + off, idesc, ks > 0);
+            const uint64_t offa = (uint64_t)(((ks >> 2) * 128 * 128 + (ks & 3) * 32) >> 4);
+            const uint64_t offb = (uint64_t)(((ks >> 2) * NC * 128 + (ks & 3) * 32) >> 4);
+            umma_bf16(d, ad0 + offa, bd0 + offb, idesc, ks > 0);
           }
+          umma_commit(smem_u32(&acc_full[slot]));      // this accumulator is complete
         }
-        umma_commit(smem_u32(&acc_full[b]));       // the accumulators of this column tile are complete
-        umma_commit(smem_u32(&b_empty[br.i]));     // ... and its stage has been read
+        if (ok) umma_commit(smem_u32(&b_empty[br.i])); // ... and the tile's stage has been read
         br.next(NST);
       }
-      if (ok) umma_commit(smem_u32(a_empty));      // the unit's rows have been read
+      if (ok) umma_commit(smem_u32(a_empty));          // the unit's rows have been read
       ++nu;
       t += took;
     }
-  } else if (warp >= 8) {
-    // ---------------- reduce: thread = one row of the unit (its tensor-memory lane) ----------------
-    const int h = (warp - 8) >> 2, quarter = warp & 3, R = quarter * 32 + lane;
-    const uint32_t trow0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)h * 128;
-    int uacc = 0, jr = 0;
+  } else if (warp >= 4) {
+    // ---------------- reduce: warp = 32 rows (its tensor-memory lanes) x one half of the 256 columns ----------------
+    const int quarter = warp & 3, part = (warp - 4) >> 2, R = quarter * 32 + lane;
+    const uint32_t trow0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(part * 128);
+    int item = 0, jr = 0, nu = 0;
     bool ok = true;
     for (int t = t0; t < t1 && ok;) {
       const int took = rkv_unit(c, t, t1, w, u);
-      const int row = u.row0 + h * 128 + R;
-      const bool live = h < u.halves && row < w.n;
-      const float rn_i = live ? __ldg(rn + (size_t)w.seg * c.cap + row) : 0.f;
-      const int jdiag = (u.row0 + h * 128) >> 7;   // the column tile that holds this warpgroup's diagonal
-      float m = -INFINITY;
-      for (int j = 0; j < u.ntj; ++j, ++uacc) {
-        const int b = uacc & 1;
-        if (!mbar_wait_warp(smem_u32(&acc_full[b]), (uacc >> 1) & 1)) { set_status(c, kDevWaitTimeout); ok = false; break; }
-        tc_fence_after();
-        if (h < u.halves) {
-          const float *rj = Rn + jr * 128;
-          const int valid = min(128, w.n - j * 128);   // columns of this tile that are pairs of the segment
-          const bool plain = j != jdiag && valid == 128;
-#pragma unroll 1
-          for (int c4 = 0; c4 < 4; ++c4) {
-            uint32_t v[32];
-            tmem_ld32_issue(trow0 + (uint32_t)(b * 256 + c4 * 32), v);
-            tmem_ld_wait(v);
-            if (plain) {
+      float m[2] = {-INFINITY, -INFINITY};   // running maxima of this thread's row in each half of the unit
+      for (int j = 0; j < u.ntj && ok; ++j) {
+        const float *rj = Rn + jr * NC + part * 128;
+        const int col0 = j * NC + part * 128;                  // first column of this warp's share
+        const int valid = max(0, min(128, w.n - col0));        // columns of it that are pairs of the segment
 #pragma unroll
-              for (int k = 0; k < 32; k += 4) {
-                const float4 r4 = *reinterpret_cast<const float4 *>(rj + c4 * 32 + k);
-                m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(v[k]) * r4.x, __uint_as_float(v[k + 1]) * r4.y),
-                                   fmaxf(__uint_as_float(v[k + 2]) * r4.z, __uint_as_float(v[k + 3]) * r4.w)));
-              }
-            } else {
+        for (int h = 0; h < 2; ++h) {
+          if (h < u.halves) {
+            const int slot = item & 1;
+            if (!mbar_wait_warp(smem_u32(&acc_full[slot]), (item >> 1) & 1)) { set_status(c, kDevWaitTimeout); ok = false; break; }
+            tc_fence_after();
+            const int row = u.row0 + h * 128 + R;
+            const bool plain = valid == 128 && col0 != u.row0 + h * 128;   // no diagonal, no columns past the end
+            float mm = m[h];
+            // 32 columns at a time, the next 32 on their way from tensor memory meanwhile.
+            auto reduce32 = [&](const uint32_t (&v)[32], int c4) {
+              if (plain) {
+                float m1 = -INFINITY;
 #pragma unroll
-              for (int k = 0; k < 32; ++k) {
-                const int col = c4 * 32 + k;
-                if (col < valid && j * 128 + col != row) m = fmaxf(m, __uint_as_float(v[k]) * rj[col]);
+                for (int k = 0; k < 32; k += 4) {
+                  const float4 r4 = *reinterpret_cast<const float4 *>(rj + c4 * 32 + k);
+                  const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(v[k]), __uint_as_float(v[k + 1])), make_float2(r4.x, r4.y));
+                  const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(v[k + 2]), __uint_as_float(v[k + 3])), make_float2(r4.z, r4.w));
+                  mm = fmaxf(fmaxf(mm, p0.x), p0.y);
+                  m1 = fmaxf(fmaxf(m1, p1.x), p1.y);
+                }
+                mm = fmaxf(mm, m1);
+              } else {
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                  const int col = c4 * 32 + k;
+                  if (col < valid && col0 + col != row) mm = fmaxf(mm, __uint_as_float(v[k]) * rj[col]);
+                }
               }
+            };
+            if (valid > 0) {
+              const uint32_t tacc = trow0 + (uint32_t)(slot * NC);
+              uint32_t va[32], vb[32];
+              tmem_ld32_issue(tacc, va);
+              tmem_ld_wait(va);
+              tmem_ld32_issue(tacc + 32, vb);
+              reduce32(va, 0);
+              tmem_ld_wait(vb);
+              tmem_ld32_issue(tacc + 64, va);
+              reduce32(vb, 1);
+              tmem_ld_wait(va);
+              tmem_ld32_issue(tacc + 96, vb);
+              reduce32(va, 2);
+              tmem_ld_wait(vb);
+              reduce32(vb, 3);
             }
+            m[h] = mm;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&acc_empty[slot]));   // this warp's share of the accumulator has been read
+            ++item;
           }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[b]));   // this warp's share of the accumulators has been read
         if (++jr == NR) jr = 0;
       }
-      if (live && ok) {
-        const float s = m > -INFINITY ? rn_i * m : 0.f;        // a single pair has no other pair
-        float *o = out + (size_t)(w.seg - seg_base) * c.cap + row;
-        *o = lambda_a * *o - lambda_s * s;
+      // The two column halves of a row meet: the warps of the second half hand their maxima over.
+      float *xs = Xch + (nu & (kRkvXch - 1)) * 256;
+      if (part == 1) {
+        xs[R] = m[0];
+        xs[128 + R] = m[1];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&x_full[nu & (kRkvXch - 1)]));
+      } else if (ok) {
+        if (!mbar_wait_warp(smem_u32(&x_full[nu & (kRkvXch - 1)]), (nu / kRkvXch) & 1)) { set_status(c, kDevWaitTimeout); break; }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int row = u.row0 + h * 128 + R;
+          if (h < u.halves && row < w.n) {
+            const float mx = fmaxf(m[h], xs[h * 128 + R]);
+            const float s = mx > -INFINITY ? __ldg(rn + (size_t)w.seg * c.cap + row) * mx : 0.f;   // a single pair has no other pair
+            float *o = out + (size_t)(w.seg - seg_base) * c.cap + row;
+            *o = lambda_a * *o - lambda_s * s;
+          }
+        }
       }
+      ++nu;
       t += took;
     }
   }
