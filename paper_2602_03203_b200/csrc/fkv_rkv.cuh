@@ -38,15 +38,23 @@ constexpr int kRkvStages = 2;                 // column tiles (256 keys) in the 
 constexpr int kRkvCols = 256;                 // keys per column tile = N of the mma
 constexpr int kRkvNormSlots = kRkvStages + 2; // the copies run at most kRkvStages ahead of the mma, the mma at most one tile ahead of the reduction
 constexpr int kRkvXch = 4;                    // hand-over slots of the row maxima (by unit)
-constexpr int kRkvThreads = 12 * 32;
+constexpr int kRkvParts = 2;                  // reducing warps per 32 rows: each takes 256 / kRkvParts columns of an accumulator
+constexpr int kRkvThreads = (4 + 4 * kRkvParts) * 32;
 
 struct RkvSmem {
   static __host__ __device__ size_t tile(int D) { return (size_t)(D / 64) * 128 * 128; }   // 128 rows: [D/64][128][128 B]
   // 1 KB alignment slack | A (two tiles) | B ring (two tiles' worth a stage) | reciprocal norms | row maxima | barriers
   static __host__ __device__ size_t bytes(int D) {
-    return 1024 + (2 + 2 * kRkvStages) * tile(D) + (size_t)kRkvNormSlots * kRkvCols * 4 + (size_t)kRkvXch * 256 * 4 + 256;
+    return 1024 + (2 + 2 * kRkvStages) * tile(D) + (size_t)kRkvNormSlots * kRkvCols * 4 + (size_t)kRkvXch * (kRkvParts - 1) * 256 * 4 + 256;
   }
 };
+
+// The largest of three (one instruction).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 
 // One page's K rows, channels 64 q .. 64 q + 63, to 16 consecutive 128-byte rows of an operand tile.
 __device__ __forceinline__ void tma_page_k(uint32_t dst, const CUtensorMap *tm, int q, int page, uint32_t bar) {
@@ -125,8 +133,8 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __gri
   uint8_t *At = smem;                                        // [2][D/64][128 rows][128 B]
   uint8_t *Bt = At + 2 * tb;                                 // [NST][D/64][256 rows][128 B]
   float *Rn = reinterpret_cast<float *>(Bt + NST * 2 * tb);  // [NR][256]
-  float *Xch = Rn + NR * NC;                                 // [kRkvXch][2 halves][128 rows]
-  uint64_t *bars = reinterpret_cast<uint64_t *>(Xch + kRkvXch * 256);
+  float *Xch = Rn + NR * NC;                                 // [kRkvXch][kRkvParts - 1][2 halves][128 rows]
+  uint64_t *bars = reinterpret_cast<uint64_t *>(Xch + kRkvXch * (kRkvParts - 1) * 256);
   uint64_t *a_full = bars, *a_empty = bars + 1, *b_full = bars + 2, *b_empty = b_full + NST;
   uint64_t *acc_full = b_empty + NST, *acc_empty = acc_full + 2, *x_full = acc_empty + 2;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(x_full + kRkvXch);
@@ -135,8 +143,8 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __gri
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(a_full), 1); mbar_init(smem_u32(a_empty), 1);
     for (int s = 0; s < NST; ++s) { mbar_init(smem_u32(&b_full[s]), 1); mbar_init(smem_u32(&b_empty[s]), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&acc_full[b]), 1); mbar_init(smem_u32(&acc_empty[b]), 8); }
-    for (int x = 0; x < kRkvXch; ++x) mbar_init(smem_u32(&x_full[x]), 4);
+    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&acc_full[b]), 1); mbar_init(smem_u32(&acc_empty[b]), 4 * kRkvParts); }
+    for (int x = 0; x < kRkvXch; ++x) mbar_init(smem_u32(&x_full[x]), 4 * (kRkvParts - 1));
     fence_barrier_init();
   }
   tc_fence_before();
@@ -237,17 +245,18 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __gri
     }
   } else if (warp >= 4) {
     // ---------------- reduce: warp = 32 rows (its tensor-memory lanes) x one half of the 256 columns ----------------
+    constexpr int CW = NC / kRkvParts, NCHUNK = CW / 32;   // this warp's columns of an accumulator
     const int quarter = warp & 3, part = (warp - 4) >> 2, R = quarter * 32 + lane;
-    const uint32_t trow0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(part * 128);
+    const uint32_t trow0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(part * CW);
     int item = 0, jr = 0, nu = 0;
     bool ok = true;
     for (int t = t0; t < t1 && ok;) {
       const int took = rkv_unit(c, t, t1, w, u);
       float m[2] = {-INFINITY, -INFINITY};   // running maxima of this thread's row in each half of the unit
       for (int j = 0; j < u.ntj && ok; ++j) {
-        const float *rj = Rn + jr * NC + part * 128;
-        const int col0 = j * NC + part * 128;                  // first column of this warp's share
-        const int valid = max(0, min(128, w.n - col0));        // columns of it that are pairs of the segment
+        const float *rj = Rn + jr * NC + part * CW;
+        const int col0 = j * NC + part * CW;                   // first column of this warp's share
+        const int valid = max(0, min(CW, w.n - col0));         // columns of it that are pairs of the segment
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           if (h < u.halves) {
@@ -255,7 +264,7 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __gri
             if (!mbar_wait_warp(smem_u32(&acc_full[slot]), (item >> 1) & 1)) { set_status(c, kDevWaitTimeout); ok = false; break; }
             tc_fence_after();
             const int row = u.row0 + h * 128 + R;
-            const bool plain = valid == 128 && col0 != u.row0 + h * 128;   // no diagonal, no columns past the end
+            const bool plain = valid == CW && (col0 & ~127) != u.row0 + h * 128;   // no diagonal, no columns past the end
             float mm = m[h];
             // 32 columns at a time, the next 32 on their way from tensor memory meanwhile.
             auto reduce32 = [&](const uint32_t (&v)[32], int c4) {
@@ -266,8 +275,8 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __gri
                   const float4 r4 = *reinterpret_cast<const float4 *>(rj + c4 * 32 + k);
                   const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(v[k]), __uint_as_float(v[k + 1])), make_float2(r4.x, r4.y));
                   const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(v[k + 2]), __uint_as_float(v[k + 3])), make_float2(r4.z, r4.w));
-                  mm = fmaxf(fmaxf(mm, p0.x), p0.y);
-                  m1 = fmaxf(fmaxf(m1, p1.x), p1.y);
+                  mm = max3(mm, p0.x, p0.y);
+                  m1 = max3(m1, p1.x, p1.y);
                 }
                 mm = fmaxf(mm, m1);
               } else {
@@ -282,17 +291,15 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __gri
               const uint32_t tacc = trow0 + (uint32_t)(slot * NC);
               uint32_t va[32], vb[32];
               tmem_ld32_issue(tacc, va);
-              tmem_ld_wait(va);
-              tmem_ld32_issue(tacc + 32, vb);
-              reduce32(va, 0);
-              tmem_ld_wait(vb);
-              tmem_ld32_issue(tacc + 64, va);
-              reduce32(vb, 1);
-              tmem_ld_wait(va);
-              tmem_ld32_issue(tacc + 96, vb);
-              reduce32(va, 2);
-              tmem_ld_wait(vb);
-              reduce32(vb, 3);
+#pragma unroll
+              for (int cc = 0; cc < NCHUNK; cc += 2) {
+                tmem_ld_wait(va);
+                tmem_ld32_issue(tacc + (uint32_t)(cc * 32 + 32), vb);
+                reduce32(va, cc);
+                tmem_ld_wait(vb);
+                if (cc + 2 < NCHUNK) tmem_ld32_issue(tacc + (uint32_t)(cc * 32 + 64), va);
+                reduce32(vb, cc + 1);
+              }
             }
             m[h] = mm;
             tc_fence_before();
@@ -303,11 +310,11 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __gri
         }
         if (++jr == NR) jr = 0;
       }
-      // The two column halves of a row meet: the warps of the second half hand their maxima over.
-      float *xs = Xch + (nu & (kRkvXch - 1)) * 256;
-      if (part == 1) {
-        xs[R] = m[0];
-        xs[128 + R] = m[1];
+      // The column parts of a row meet: the warps of the other parts hand their maxima over.
+      float *xs = Xch + (nu & (kRkvXch - 1)) * (kRkvParts - 1) * 256;
+      if (part > 0) {
+        xs[(part - 1) * 256 + R] = m[0];
+        xs[(part - 1) * 256 + 128 + R] = m[1];
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&x_full[nu & (kRkvXch - 1)]));
       } else if (ok) {
@@ -316,7 +323,9 @@ __global__ void __launch_bounds__(kRkvThreads, 1) k_rkv_score(Ctx c, const __gri
         for (int h = 0; h < 2; ++h) {
           const int row = u.row0 + h * 128 + R;
           if (h < u.halves && row < w.n) {
-            const float mx = fmaxf(m[h], xs[h * 128 + R]);
+            float mx = m[h];
+#pragma unroll
+            for (int q = 0; q < kRkvParts - 1; ++q) mx = fmaxf(mx, xs[q * 256 + h * 128 + R]);
             const float s = mx > -INFINITY ? __ldg(rn + (size_t)w.seg * c.cap + row) * mx : 0.f;   // a single pair has no other pair
             float *o = out + (size_t)(w.seg - seg_base) * c.cap + row;
             *o = lambda_a * *o - lambda_s * s;
