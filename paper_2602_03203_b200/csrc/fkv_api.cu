@@ -326,11 +326,30 @@ int launch_rkv_t(fkv_cache *c, float *out, int seg_base, int max_old, int nwork_
   k_rkv_prepare<D><<<dim3(nwork_bound, (max_old + 127) / 128), 128, 0, st>>>(c->ctx, out, rn, seg_base,
                                                                              FKV_FEATURE_WINDOW8);
   FKV_LAUNCHED(c);
-  const size_t smem = RkvSmem::bytes(D);
-  static SmemOptIn opt_in;
-  FKV_CUDA(opt_in.ensure(k_rkv_score<D>, smem));
-  const int grid = (int)std::max<long long>(1, std::min<long long>(c->sm_count, tiles));
-  k_rkv_score<D><<<grid, kRkvThreads, smem, st>>>(c->ctx, c->k_rows, out, rn, seg_base, la, ls);
+  if (tiles > 4) {
+    // Pairs of CTAs that multiply as one (a unit is up to four tiles).
+    const size_t smem = RkvPairSmem::bytes(D);
+    static SmemOptIn opt_in;
+    FKV_CUDA(opt_in.ensure(k_rkv_score_pair<D>, smem));
+    const int npairs = (int)std::max<long long>(1, std::min<long long>(c->sm_count / 2, (tiles + 3) / 4));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * npairs);
+    cfg.blockDim = dim3(kRkvThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    FKV_CUDA(cudaLaunchKernelEx(&cfg, k_rkv_score_pair<D>, c->ctx, c->k_rows, out, (const float *)rn, seg_base, la, ls));
+  } else {
+    const size_t smem = RkvSmem::bytes(D);
+    static SmemOptIn opt_in;
+    FKV_CUDA(opt_in.ensure(k_rkv_score<D>, smem));
+    const int grid = (int)std::max<long long>(1, std::min<long long>(c->sm_count, tiles));
+    k_rkv_score<D><<<grid, kRkvThreads, smem, st>>>(c->ctx, c->k_rows, out, rn, seg_base, la, ls);
+  }
   FKV_LAUNCHED(c);
   return FKV_OK;
 }
