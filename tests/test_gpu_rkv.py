@@ -1,9 +1,10 @@
 """The R-KV baseline score (Appendix E.2) on the GPU against the CPU oracle, through the C ABI.
 
-The score's similarity term is the n x n contraction of a segment's keys on the tensor cores; the
-cases span one pair, lengths around the 128-row operand tiles and the 256-row units, ragged last
-tiles, several segments of different lengths per launch, both head dimensions, duplicate and zero
-keys.  Tolerance: 1e-3 on the scores (the figure every score of this library is held to); selection and
+The score's similarity term is the n x n contraction of a segment's keys on the tensor cores (pairs of
+CTAs that multiply as one; single CTAs for launches of four tiles or fewer); the cases span one pair,
+lengths around the 128-row operand tiles and the units of two and four tiles, ragged last tiles, several
+segments of different lengths per launch, ranges of CTA pairs that cut through segments, both head
+dimensions, duplicate and zero keys.  Tolerance: 1e-3 on the scores (the figure every score of this library is held to); selection and
 compaction from the GPU's own scores are bit-exact.
 """
 import numpy as np
@@ -38,6 +39,25 @@ def test_rkv_scores_match_oracle(lens, g, D, Hkv):
                 # similarity weight 0: the SnapKV score, bit for bit
                 assert np.array_equal(snap[s, h, :n], oracle.score_feature(A, g, oracle.SNAPKV_COLUMN))
     assert worst <= SCORE_TOL, worst
+    assert ld.cache.device_status()[0] == 0
+
+
+def test_rkv_pairs_of_ctas_with_ragged_ranges():
+    # 332 tiles over 74 pairs of CTAs: five tiles a pair, so units of four tiles and of one, ranges that start and
+    # end in the middle of segments, pairs whose second CTA has no rows.  Sampled rows: the oracle takes them one by
+    # one (first and last rows, unit and tile boundaries of each segment, random ones).
+    lens = (9000, 7000, 5000)
+    w = wl.Workload("rkv_pairs", 1, 2, 4, 128, lens, tuple(1 << 20 for _ in lens), 0, 57, "channel_lognormal")
+    ld = Loaded(w)
+    got = npf(ld.cache.score_rkv(0))
+    rng = np.random.default_rng(11)
+    for s, n in enumerate(lens):
+        rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, 383, 384, 511, 512, 639, 640, n - 129, n - 128, n - 1],
+                                         rng.integers(0, n, 120)])).astype(np.int32)
+        for h in range(w.num_kv_heads):
+            K, V, A, _ = ld.head(0, s, h)
+            ref = oracle.score_rkv(K, A, w.group_size, rows=rows)
+            assert np.abs(got[s, h, rows] - ref).max() <= SCORE_TOL, (s, h)
     assert ld.cache.device_status()[0] == 0
 
 
