@@ -18,9 +18,10 @@
 //               (the tensor map sees the page pool as [page][row][64-channel half][64 channels]), 2 KB that land as
 //               16 rows of a K-major operand tile - the page record's swizzle is the shared-memory swizzle.  A lane
 //               per copy: the unit's 256 rows once, then the column tiles into a ring, with their reciprocal norms;
-//   warp 1      one lane issues tcgen05.mma (bf16 x bf16 -> fp32, M = 128, N = 256, K = 16 per instruction: an
-//               instruction takes about 130 cycles whatever its N up to 128, and 155 at N = 256) into one of the
-//               two 256-column accumulators of tensor memory and hands them on with tcgen05.commit;
+//   warp 1      one lane issues tcgen05.mma (bf16 x bf16 -> fp32, M = 128, N = 256, K = 16 per instruction: wide
+//               accumulators mean few hand-overs per product, and the hand-over round trip is what tensor memory's
+//               room for two of them cannot hide) into one of the two 256-column accumulators and hands them on
+//               with tcgen05.commit;
 //   warps 4-11  reduce: warp = 32 rows (its tensor-memory lanes) x 128 of the 256 columns; a thread scales the
 //               products by the column's reciprocal norm and keeps the running maximum of its row, the next 32
 //               columns on their way from tensor memory meanwhile; the diagonal and the columns past the segment's
