@@ -23,7 +23,8 @@ SCORE_TOL = 1e-3
 
 @pytest.mark.parametrize("lens,g,D,Hkv", [((1, 2), 4, 64, 2), ((100, 128), 4, 128, 2), ((129, 255), 1, 128, 1),
                                           ((256, 257), 7, 128, 2), ((300, 700, 1000, 17), 4, 128, 2),
-                                          ((1500,), 8, 64, 3), ((2049, 640), 2, 128, 4)])
+                                          ((1500,), 8, 64, 3), ((2049, 640), 2, 128, 4),
+                                          ((512, 513, 1024, 1025), 2, 128, 1), ((511, 769), 4, 64, 2)])
 def test_rkv_scores_match_oracle(lens, g, D, Hkv):
     w = wl.Workload("rkv", 2, Hkv, g, D, lens, tuple(1 << 20 for _ in lens), 0, 51, "channel_lognormal")
     ld = Loaded(w)
