@@ -214,6 +214,9 @@ int fkv_evict_by_feature(fkv_cache *c, int layer, int32_t column, void *stream);
  * No normalisation of either term.  Cost: the n x n products of a segment's keys, 2 n^2 D flops, on the tensor
  * cores.  Features must be finite.  Everything else is as in fkv_evict_by_feature.  FKV_RKV_LAMBDA_* are the
  * paper's weights.  fkv_score_rkv is the score alone (layout as fkv_score).
+ * Errors beyond those of fkv_evict_by_feature: FKV_ERR_CUDA if the driver's tensor-map encoder cannot be reached or
+ * refuses the page pool's geometry, or if the device cannot place clusters of two thread blocks (the contraction
+ * runs on pairs of SMs); fkv_last_cuda_error has the text.  Nothing of the cache is changed in that case.
  */
 #define FKV_RKV_LAMBDA_ATTN 0.1f
 #define FKV_RKV_LAMBDA_SIM 0.9f
