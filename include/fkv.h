@@ -216,7 +216,7 @@ int fkv_evict_by_feature(fkv_cache *c, int layer, int32_t column, void *stream);
  * paper's weights.  fkv_score_rkv is the score alone (layout as fkv_score).
  * Errors beyond those of fkv_evict_by_feature: FKV_ERR_CUDA if the driver's tensor-map encoder cannot be reached or
  * refuses the page pool's geometry, or if the device cannot place clusters of two thread blocks (the contraction
- * runs on pairs of SMs); fkv_last_cuda_error has the text.  Nothing of the cache is changed in that case.
+ * runs on pairs of SMs); fkv_last_cuda_error has the text.  No pair is evicted or moved in that case.
  */
 #define FKV_RKV_LAMBDA_ATTN 0.1f
 #define FKV_RKV_LAMBDA_SIM 0.9f
